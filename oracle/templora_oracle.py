@@ -1,0 +1,150 @@
+"""fp64 CPU oracle for the Temp-Lora chunk-update hot path.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition that the
+CUDA library is checked against.  It shares no code with the CUDA path and is
+imported only by the tests, by the smoke check and by the CPU-baseline leg of
+the benchmark.  The product never calls it.
+
+What it computes (Temp-Lora, Section "Temp-Lora" and Algorithm 1, step
+"Train Theta_k ... (n epochs, learning rate alpha)"; the module is the LoRA
+module of Hu et al. that the paper adopts by citation, with the hyper-parameters
+of the paper's "Setup" paragraph: alpha = 64, rank = 64, learning rate 5e-5,
+n = 2 epochs, bfloat16 training):
+
+    U  = x A^T                         [T, r]
+    y  = x W0^T + s U B^T              [T, d_out]         s = alpha / r
+    V  = dY B                          [T, r]
+    dX = dY W0 + s V A                 [T, d_in]
+    dB = s dY^T U                      [d_out, r]
+    dA = s V^T x                       [r, d_in]
+    (W0 is frozen: the method never alters the base model, so no dW0 exists.)
+
+Every function is the definition written out with numpy matmuls on float64
+arrays, in the order above; nothing is blocked, fused or reordered.
+
+Pins (tests/test_oracle_pins.py): brute-force Python loops on tiny shapes, an
+integer worked example under tests/golden/, B = 0 reduction, the merged-weight
+identity, exact finite differences (the loss sum(dY*y) is linear in each of
+x, A, B separately), additivity of dA/dB over row partitions, the closed-form
+first AdamW step, the constant-gradient AdamW trajectory, and torch's own
+bfloat16 cast for the rounding helper.
+
+Parity with numbers printed by the paper: parity unpinned.  The paper prints no
+worked numeric example and no per-layer value for this path; the pins above are
+mathematical.
+"""
+import numpy as np
+
+F64 = np.float64
+
+
+def _f64(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=F64))
+
+
+# --------------------------------------------------------------------------
+# forward:  y = x W0^T + s (x A^T) B^T            (Temp-Lora module forward)
+# --------------------------------------------------------------------------
+def linear_fwd(x, W0, A, B, s):
+    """x [T,d_in], W0 [d_out,d_in], A [r,d_in], B [d_out,r] -> (y [T,d_out], U [T,r])."""
+    x, W0, A, B = _f64(x), _f64(W0), _f64(A), _f64(B)
+    U = x @ A.T
+    y = x @ W0.T + F64(s) * (U @ B.T)
+    return y, U
+
+
+# --------------------------------------------------------------------------
+# backward with W0 frozen (no dW0: the base model is never altered)
+# --------------------------------------------------------------------------
+def linear_bwd(x, dY, W0, A, B, s):
+    """-> (dX [T,d_in], dA [r,d_in], dB [d_out,r]); gradients are plain sums over tokens."""
+    x, dY, W0, A, B = _f64(x), _f64(dY), _f64(W0), _f64(A), _f64(B)
+    s = F64(s)
+    U = x @ A.T
+    V = dY @ B
+    dX = dY @ W0 + s * (V @ A)
+    dB = s * (dY.T @ U)
+    dA = s * (V.T @ x)
+    return dX, dA, dB
+
+
+# --------------------------------------------------------------------------
+# decode-time forward with the current module, token by token
+# (Algorithm 1, generation step  Y[i] = Theta_k(...))
+# --------------------------------------------------------------------------
+def decode_fwd(x, W0, A, B, s):
+    """x [n,d_in] (n generated-token rows) -> y [n,d_out]; one GEMV chain per token."""
+    x, W0, A, B = _f64(x), _f64(W0), _f64(A), _f64(B)
+    y = np.empty((x.shape[0], W0.shape[0]), dtype=F64)
+    for i in range(x.shape[0]):
+        u = A @ x[i]
+        y[i] = W0 @ x[i] + F64(s) * (B @ u)
+    return y
+
+
+# --------------------------------------------------------------------------
+# AdamW (decoupled weight decay, bias-corrected), step index t is 1-based
+# --------------------------------------------------------------------------
+def adamw_step(p, g, m, v, lr, beta1, beta2, eps, weight_decay, t):
+    """Returns new (p, m, v).  eps is added to sqrt(v_hat), outside the root."""
+    p, g, m, v = _f64(p), _f64(g), _f64(m), _f64(v)
+    lr, beta1, beta2, eps, wd = F64(lr), F64(beta1), F64(beta2), F64(eps), F64(weight_decay)
+    p = p * (1.0 - lr * wd)
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** int(t))
+    v_hat = v / (1.0 - beta2 ** int(t))
+    p = p - lr * m_hat / (np.sqrt(v_hat) + eps)
+    return p, m, v
+
+
+# --------------------------------------------------------------------------
+# bfloat16 storage rounding (round to nearest, ties to even) of fp32 values
+# --------------------------------------------------------------------------
+def round_bf16(a):
+    """Value of `a` after fp32 -> bfloat16 storage (RNE), returned as float64."""
+    f = np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+    bits = f.view(np.uint32).astype(np.uint64)
+    lsb = (bits >> np.uint64(16)) & np.uint64(1)
+    rounded = (bits + np.uint64(0x7FFF) + lsb) & np.uint64(0xFFFF0000)
+    out = rounded.astype(np.uint32).view(np.float32)
+    out = np.where(np.isnan(f), f, out)
+    return out.astype(F64)
+
+
+# --------------------------------------------------------------------------
+# the whole update of one block of projections: n epochs over the chunk,
+# one optimizer step per epoch (batch = chunk)
+# --------------------------------------------------------------------------
+def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf16_work=False):
+    """projs: list of dicts with keys x, dY, W0, s, A_master, B_master and optionally
+    mA, vA, mB, vB (default 0).  For each epoch: forward and backward of every
+    projection with the current working A, B; then step += 1 and AdamW on every
+    A and B.  With bf16_work the GEMMs read round_bf16(master), the optimizer
+    updates the master (fp32 master + bf16 working copy, which is what bfloat16
+    training under ZeRO-2 implies).
+
+    Returns (state, step): state[i] has A_master, B_master, mA, vA, mB, vB and the
+    last epoch's y, dX, dA, dB.
+    """
+    st = []
+    for p in projs:
+        A = _f64(p["A_master"])
+        B = _f64(p["B_master"])
+        st.append(dict(A_master=A, B_master=B,
+                       mA=_f64(p.get("mA", np.zeros_like(A))), vA=_f64(p.get("vA", np.zeros_like(A))),
+                       mB=_f64(p.get("mB", np.zeros_like(B))), vB=_f64(p.get("vB", np.zeros_like(B)))))
+    step = int(step0)
+    for _ in range(int(epochs)):
+        for p, q in zip(projs, st):
+            A = round_bf16(q["A_master"]) if bf16_work else q["A_master"]
+            B = round_bf16(q["B_master"]) if bf16_work else q["B_master"]
+            q["y"], _ = linear_fwd(p["x"], p["W0"], A, B, p["s"])
+            q["dX"], q["dA"], q["dB"] = linear_bwd(p["x"], p["dY"], p["W0"], A, B, p["s"])
+        step += 1
+        for q in st:
+            q["A_master"], q["mA"], q["vA"] = adamw_step(q["A_master"], q["dA"], q["mA"], q["vA"],
+                                                         lr, beta1, beta2, eps, weight_decay, step)
+            q["B_master"], q["mB"], q["vB"] = adamw_step(q["B_master"], q["dB"], q["mB"], q["vB"],
+                                                         lr, beta1, beta2, eps, weight_decay, step)
+    return st, step

@@ -1,0 +1,334 @@
+"""Pins for the fp64 oracle: it is checked against things other than itself.
+
+Brute-force scalar loops, a hand-worked integer example, algebraic identities
+of the LoRA-augmented projection, exact finite differences, and closed forms of
+AdamW.  The last test plants plausible mistakes in copies of the oracle and
+requires that the pins catch each of them.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from conftest import load_golden
+from oracle import templora_oracle as orc
+
+RNG = np.random.default_rng(1234)
+
+
+def rnd(*shape):
+    return RNG.standard_normal(shape)
+
+
+# ----------------------------------------------------------------- brute force
+def brute_fwd(x, W0, A, B, s):
+    T, d_in = x.shape
+    d_out, r = B.shape
+    y = [[0.0] * d_out for _ in range(T)]
+    for t in range(T):
+        u = [sum(x[t][k] * A[j][k] for k in range(d_in)) for j in range(r)]
+        for o in range(d_out):
+            base = sum(x[t][k] * W0[o][k] for k in range(d_in))
+            low = sum(u[j] * B[o][j] for j in range(r))
+            y[t][o] = base + s * low
+    return np.array(y)
+
+
+def brute_bwd(x, dY, W0, A, B, s):
+    T, d_in = x.shape
+    d_out, r = B.shape
+    dX = np.zeros((T, d_in)); dA = np.zeros((r, d_in)); dB = np.zeros((d_out, r))
+    for t in range(T):
+        u = [sum(x[t][k] * A[j][k] for k in range(d_in)) for j in range(r)]
+        v = [sum(dY[t][o] * B[o][j] for o in range(d_out)) for j in range(r)]
+        for k in range(d_in):
+            dX[t][k] = sum(dY[t][o] * W0[o][k] for o in range(d_out)) + s * sum(v[j] * A[j][k] for j in range(r))
+        for o in range(d_out):
+            for j in range(r):
+                dB[o][j] += s * dY[t][o] * u[j]
+        for j in range(r):
+            for k in range(d_in):
+                dA[j][k] += s * v[j] * x[t][k]
+    return dX, dA, dB
+
+
+SHAPES = [(5, 7, 6, 3), (1, 4, 9, 2), (9, 3, 2, 5)]
+
+
+@pytest.mark.parametrize("T,d_in,d_out,r", SHAPES)
+def test_fwd_bwd_match_scalar_loops(T, d_in, d_out, r):
+    x, W0, A, B, dY = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r), rnd(T, d_out)
+    s = 1.75
+    y, U = orc.linear_fwd(x, W0, A, B, s)
+    np.testing.assert_allclose(y, brute_fwd(x, W0, A, B, s), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(U, x @ A.T, rtol=1e-13, atol=1e-13)
+    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, s)
+    bX, bA, bB = brute_bwd(x, dY, W0, A, B, s)
+    np.testing.assert_allclose(dX, bX, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dA, bA, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dB, bB, rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------ worked example
+def test_hand_worked_integer_case():
+    g = load_golden("lora_integer_case.txt")
+    s = float(g["s"][0, 0])
+    y, U = orc.linear_fwd(g["x"], g["W0"], g["A"], g["B"], s)
+    assert np.array_equal(y, g["y"]) and np.array_equal(U, g["U"])
+    dX, dA, dB = orc.linear_bwd(g["x"], g["dY"], g["W0"], g["A"], g["B"], s)
+    assert np.array_equal(dX, g["dX"]) and np.array_equal(dA, g["dA"]) and np.array_equal(dB, g["dB"])
+    assert np.array_equal(orc.decode_fwd(g["x"], g["W0"], g["A"], g["B"], s), g["y"])
+
+
+# ----------------------------------------------------------------- identities
+def test_zero_B_reduces_to_base_linear_exactly():
+    T, d_in, d_out, r = 6, 11, 5, 4
+    x, W0, A, dY = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(T, d_out)
+    B = np.zeros((d_out, r))
+    y, _ = orc.linear_fwd(x, W0, A, B, 2.0)
+    assert np.array_equal(y, x @ W0.T)          # bit for bit
+    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, 2.0)
+    assert np.array_equal(dX, dY @ W0)
+    assert not dA.any()                         # no gradient reaches A through B = 0
+    assert np.abs(dB).max() > 0
+    # A = 0 kills dB and the low-rank part of dX
+    dX2, dA2, dB2 = orc.linear_bwd(x, dY, W0, np.zeros_like(A), rnd(d_out, r), 2.0)
+    assert not dB2.any() and np.array_equal(dX2, dY @ W0)
+
+
+def test_merged_weight_identity():
+    T, d_in, d_out, r, s = 8, 13, 10, 4, 2.0
+    x, W0, A, B, dY = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r), rnd(T, d_out)
+    Wm = W0 + s * (B @ A)
+    y, _ = orc.linear_fwd(x, W0, A, B, s)
+    dX, _, _ = orc.linear_bwd(x, dY, W0, A, B, s)
+    np.testing.assert_allclose(y, x @ Wm.T, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dX, dY @ Wm, rtol=1e-12, atol=1e-12)
+
+
+def test_linear_in_s():
+    T, d_in, d_out, r = 4, 6, 5, 3
+    x, W0, A, B = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r)
+    y0, _ = orc.linear_fwd(x, W0, A, B, 0.0)
+    y1, _ = orc.linear_fwd(x, W0, A, B, 1.0)
+    y3, _ = orc.linear_fwd(x, W0, A, B, 3.0)
+    np.testing.assert_allclose(y3 - y0, 3.0 * (y1 - y0), rtol=1e-12, atol=1e-12)
+
+
+def _loss(x, W0, A, B, s, dY):
+    y, _ = orc.linear_fwd(x, W0, A, B, s)
+    return float((dY * y).sum())
+
+
+def test_gradients_match_exact_finite_differences():
+    # L = sum(dY * y) is linear in each of x, A, B taken alone, so a central
+    # difference with ANY step is exact up to rounding.
+    T, d_in, d_out, r, s, h = 5, 7, 6, 3, 2.0, 0.5
+    x, W0, A, B, dY = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r), rnd(T, d_out)
+    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, s)
+
+    def fd(arr, which):
+        g = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            plus, minus = arr.copy(), arr.copy()
+            plus[idx] += h; minus[idx] -= h
+            args_p = dict(x=x, A=A, B=B); args_m = dict(x=x, A=A, B=B)
+            args_p[which] = plus; args_m[which] = minus
+            g[idx] = (_loss(args_p["x"], W0, args_p["A"], args_p["B"], s, dY)
+                      - _loss(args_m["x"], W0, args_m["A"], args_m["B"], s, dY)) / (2 * h)
+        return g
+
+    for got, ref in ((dX, fd(x, "x")), (dA, fd(A, "A")), (dB, fd(B, "B"))):
+        assert np.abs(got - ref).max() <= 1e-9 * max(1.0, np.abs(ref).max())
+
+
+def test_dA_dB_additive_over_row_partitions():
+    T, d_in, d_out, r, s = 11, 6, 7, 3, 2.0
+    x, W0, A, B, dY = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r), rnd(T, d_out)
+    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, s)
+    cut = 4
+    dX1, dA1, dB1 = orc.linear_bwd(x[:cut], dY[:cut], W0, A, B, s)
+    dX2, dA2, dB2 = orc.linear_bwd(x[cut:], dY[cut:], W0, A, B, s)
+    np.testing.assert_allclose(dA, dA1 + dA2, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dB, dB1 + dB2, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dX, np.vstack([dX1, dX2]), rtol=1e-13, atol=1e-13)
+
+
+def test_decode_equals_rows_of_chunk_forward():
+    d_in, d_out, r, s = 24, 17, 4, 2.0
+    W0, A, B = rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r)
+    for n in (1, 4, 16):
+        x = rnd(n, d_in)
+        y, _ = orc.linear_fwd(x, W0, A, B, s)
+        np.testing.assert_allclose(orc.decode_fwd(x, W0, A, B, s), y, rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------------- AdamW
+def test_adamw_hand_worked_first_step():
+    g = {k: float(v[0, 0]) for k, v in load_golden("adamw_first_step.txt").items()}
+    p, m, v = orc.adamw_step([g["p0"]], [g["g"]], [0.0], [0.0], g["lr"], g["beta1"], g["beta2"],
+                             g["eps"], g["wd"], 1)
+    assert abs(p[0] - g["p1"]) < 1e-15
+    assert abs(m[0] - g["m1"]) < 1e-16 and abs(v[0] - g["v1"]) < 1e-18
+
+
+def test_adamw_first_step_closed_form():
+    p0, g = rnd(50), rnd(50)
+    lr, b1, b2, eps, wd = 3e-3, 0.9, 0.999, 1e-8, 0.05
+    p, m, v = orc.adamw_step(p0, g, np.zeros(50), np.zeros(50), lr, b1, b2, eps, wd, 1)
+    np.testing.assert_allclose(p, p0 * (1 - lr * wd) - lr * g / (np.abs(g) + eps), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(m, (1 - b1) * g, rtol=1e-13)
+    np.testing.assert_allclose(v, (1 - b2) * g * g, rtol=1e-12)
+
+
+def test_adamw_zero_gradient_leaves_parameters():
+    p0 = rnd(20)
+    p, m, v = orc.adamw_step(p0, np.zeros(20), np.zeros(20), np.zeros(20), 5e-5, 0.9, 0.999, 1e-8, 0.0, 1)
+    assert np.array_equal(p, p0) and not m.any() and not v.any()
+
+
+def test_adamw_constant_gradient_trajectory():
+    # with a constant gradient m_hat = g and v_hat = g^2 at every step, so
+    # p_k = p0 - k lr g / (|g| + eps): pins the bias correction for t > 1
+    p0, g = rnd(30), rnd(30)
+    lr, eps = 1e-3, 1e-8
+    p, m, v = p0.copy(), np.zeros(30), np.zeros(30)
+    for t in range(1, 8):
+        p, m, v = orc.adamw_step(p, g, m, v, lr, 0.9, 0.999, eps, 0.0, t)
+        np.testing.assert_allclose(p, p0 - t * lr * g / (np.abs(g) + eps), rtol=1e-10, atol=1e-13)
+
+
+def test_adamw_sign_antisymmetry_and_torch():
+    p0, g = rnd(40), rnd(40)
+    a = orc.adamw_step(p0, g, np.zeros(40), np.zeros(40), 1e-3, 0.9, 0.999, 1e-8, 0.0, 1)[0]
+    b = orc.adamw_step(-p0, -g, np.zeros(40), np.zeros(40), 1e-3, 0.9, 0.999, 1e-8, 0.0, 1)[0]
+    np.testing.assert_allclose(a, -b, rtol=1e-14)
+    # an independent implementation: torch.optim.AdamW in float64, several steps, wd != 0
+    tp = torch.tensor(p0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.AdamW([tp], lr=2e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.1)
+    p, m, v = p0.copy(), np.zeros(40), np.zeros(40)
+    for t in range(1, 5):
+        gt = g * t
+        tp.grad = torch.tensor(gt, dtype=torch.float64)
+        opt.step()
+        p, m, v = orc.adamw_step(p, gt, m, v, 2e-3, 0.9, 0.999, 1e-8, 0.1, t)
+        np.testing.assert_allclose(p, tp.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------------- rounding
+def test_round_bf16_matches_torch_cast():
+    vals = np.concatenate([rnd(5000).astype(np.float32) * np.float32(10.0 ** RNG.integers(-6, 6)),
+                           np.array([0.0, -0.0, 1.0, 1.00390625, 1.0078125, 3.0e38, 1e-40, -1e-40,
+                                     np.inf, -np.inf], dtype=np.float32)])
+    # exact ties: mantissa bit pattern xxxx 1000 0000 0000 0000
+    ties = (np.arange(256, dtype=np.uint32) << np.uint32(16) | np.uint32(0x3F800000) | np.uint32(0x8000)).view(np.float32)
+    vals = np.concatenate([vals, ties])
+    ref = torch.from_numpy(vals).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(orc.round_bf16(vals), ref)
+
+
+# --------------------------------------------------------------- update_block
+def _mk_proj(T, d_in, d_out, r, s):
+    return dict(x=rnd(T, d_in), dY=rnd(T, d_out), W0=rnd(d_out, d_in) / math.sqrt(d_in), s=s,
+                A_master=rnd(r, d_in) * 0.1, B_master=rnd(d_out, r) * 0.1)
+
+
+def test_update_block_single_epoch_is_the_composition():
+    projs = [_mk_proj(6, 8, 5, 2, 2.0), _mk_proj(6, 5, 9, 2, 2.0)]
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    st, step = orc.update_block(projs, 1, **hp)
+    assert step == 1
+    for p, q in zip(projs, st):
+        dX, dA, dB = orc.linear_bwd(p["x"], p["dY"], p["W0"], p["A_master"], p["B_master"], p["s"])
+        A1, mA, vA = orc.adamw_step(p["A_master"], dA, 0 * dA, 0 * dA, t=1, **hp)
+        B1, mB, vB = orc.adamw_step(p["B_master"], dB, 0 * dB, 0 * dB, t=1, **hp)
+        assert np.array_equal(q["A_master"], A1) and np.array_equal(q["B_master"], B1)
+        assert np.array_equal(q["dX"], dX) and np.array_equal(q["mA"], mA) and np.array_equal(q["vB"], vB)
+
+
+def test_update_block_two_epochs_and_zero_lr():
+    projs = [_mk_proj(7, 6, 4, 3, 2.0)]
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    st2, step = orc.update_block(projs, 2, **hp)
+    assert step == 2
+    # by hand: epoch 2 starts from epoch 1's result, moments and step carried over
+    st1, _ = orc.update_block(projs, 1, **hp)
+    p2 = [dict(projs[0], A_master=st1[0]["A_master"], B_master=st1[0]["B_master"],
+               mA=st1[0]["mA"], vA=st1[0]["vA"], mB=st1[0]["mB"], vB=st1[0]["vB"])]
+    st12, step12 = orc.update_block(p2, 1, step0=1, **hp)
+    assert step12 == 2
+    assert np.array_equal(st2[0]["A_master"], st12[0]["A_master"])
+    assert np.array_equal(st2[0]["B_master"], st12[0]["B_master"])
+    # the second epoch really sees the updated module
+    assert np.abs(st2[0]["y"] - st1[0]["y"]).max() > 0
+    # lr = 0: nothing moves, epoch 2 repeats epoch 1
+    hp0 = dict(hp, lr=0.0)
+    a, _ = orc.update_block(projs, 1, **hp0)
+    b, _ = orc.update_block(projs, 2, **hp0)
+    assert np.array_equal(a[0]["y"], b[0]["y"]) and np.array_equal(a[0]["dA"], b[0]["dA"])
+    assert np.array_equal(b[0]["A_master"], projs[0]["A_master"])
+
+
+def test_update_block_bf16_working_copy():
+    projs = [_mk_proj(4, 8, 8, 2, 2.0)]
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    st, _ = orc.update_block(projs, 1, bf16_work=True, **hp)
+    Aw, Bw = orc.round_bf16(projs[0]["A_master"]), orc.round_bf16(projs[0]["B_master"])
+    y, _ = orc.linear_fwd(projs[0]["x"], projs[0]["W0"], Aw, Bw, 2.0)
+    assert np.array_equal(st[0]["y"], y)
+    # the optimizer moves the un-rounded master
+    _, dA, _ = orc.linear_bwd(projs[0]["x"], projs[0]["dY"], projs[0]["W0"], Aw, Bw, 2.0)
+    A1, _, _ = orc.adamw_step(projs[0]["A_master"], dA, 0 * dA, 0 * dA, t=1, **hp)
+    assert np.array_equal(st[0]["A_master"], A1)
+
+
+# -------------------------------------------- the pins catch planted mistakes
+def _pins_pass(fwd, bwd):
+    g = load_golden("lora_integer_case.txt")
+    s = float(g["s"][0, 0])
+    try:
+        y, _ = fwd(g["x"], g["W0"], g["A"], g["B"], s)
+        dX, dA, dB = bwd(g["x"], g["dY"], g["W0"], g["A"], g["B"], s)
+        ok = all(np.array_equal(a, b) for a, b in ((y, g["y"]), (dX, g["dX"]), (dA, g["dA"]), (dB, g["dB"])))
+        T, d_in, d_out, r = 5, 7, 6, 3
+        rs = np.random.default_rng(7)
+        x, W0, A, B, dY = (rs.standard_normal(sh) for sh in ((T, d_in), (d_out, d_in), (r, d_in), (d_out, r), (T, d_out)))
+        y, _ = fwd(x, W0, A, B, 1.5)
+        dX, dA, dB = bwd(x, dY, W0, A, B, 1.5)
+        bX, bA, bB = brute_bwd(x, dY, W0, A, B, 1.5)
+        ok = ok and np.allclose(y, brute_fwd(x, W0, A, B, 1.5), rtol=1e-11, atol=1e-11)
+        ok = ok and np.allclose(dX, bX, rtol=1e-11, atol=1e-11) and np.allclose(dA, bA, rtol=1e-11, atol=1e-11)
+        ok = ok and np.allclose(dB, bB, rtol=1e-11, atol=1e-11)
+        return bool(ok)
+    except Exception:
+        return False
+
+
+def test_pins_catch_planted_mistakes():
+    assert _pins_pass(orc.linear_fwd, orc.linear_bwd)
+    f, b = orc.linear_fwd, orc.linear_bwd
+    wrong_fwd = [
+        lambda x, W0, A, B, s: (x @ W0.T + (x @ A.T) @ B.T, x @ A.T),               # dropped s
+        lambda x, W0, A, B, s: (x @ W0.T - s * (x @ A.T) @ B.T, x @ A.T),           # wrong sign
+        lambda x, W0, A, B, s: (x @ W0.T + s * s * (x @ A.T) @ B.T, x @ A.T),       # s applied twice
+        lambda x, W0, A, B, s: (x @ W0.T, x @ A.T),                                  # dropped term
+    ]
+    for wf in wrong_fwd:
+        assert not _pins_pass(wf, b)
+
+    def bwd_variant(kind):
+        def fn(x, dY, W0, A, B, s):
+            U, V = x @ A.T, dY @ B
+            dX = dY @ W0 + s * (V @ A)
+            dB = s * (dY.T @ U)
+            dA = s * (V.T @ x)
+            if kind == "dX_no_lora": dX = dY @ W0
+            if kind == "dB_no_s": dB = dY.T @ U
+            if kind == "dA_uses_U": dA = s * (U.T @ x)
+            if kind == "dB_uses_V": dB = s * (dY.T @ V)
+            if kind == "dA_mean": dA = dA / x.shape[0]
+            return dX, dA, dB
+        return fn
+    for kind in ("dX_no_lora", "dB_no_s", "dA_uses_U", "dB_uses_V", "dA_mean"):
+        assert not _pins_pass(f, bwd_variant(kind))

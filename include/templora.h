@@ -1,0 +1,169 @@
+/*
+ * templora.h -- C ABI of the B200 (sm_100a) Temp-Lora chunk-update library.
+ *
+ * The library runs the per-chunk inference-time update of a temporary LoRA
+ * module ("Train Theta_k: In X_T -> Out Chunk_k (n epochs, learning rate alpha)",
+ * Algorithm 1 of the Temp-Lora paper) for LoRA-augmented linear projections, and
+ * the decode-time forward used between updates (Algorithm 1, generation step).
+ *
+ * Notation (row-major, contiguous rows, no bias):
+ *     x  [T, d_in]       chunk activations           W0 [d_out, d_in]  frozen base weight
+ *     A  [r, d_in]       LoRA down-projection        B  [d_out, r]     LoRA up-projection
+ *     y, dY [T, d_out]   output / upstream gradient  dX [T, d_in]      input gradient
+ *     U = x A^T [T, r]   V = dY B [T, r]             s = alpha / r     (paper: 64/64)
+ *
+ * General conventions
+ *   - Every data pointer is a DEVICE pointer unless stated otherwise; descriptor
+ *     arrays (templora_linear_t[], templora_param_t[], pointer arrays) are HOST arrays.
+ *   - The caller owns every buffer, the workspace included.  The library allocates
+ *     no device memory, frees nothing, never writes W0, and never synchronises the
+ *     stream (templora_read_device_status excepted).  All work is enqueued on
+ *     `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - dtype TEMPLORA_BF16: x, W0, A, B, y, dY, dX are bfloat16; products accumulate
+ *     in fp32; gradients dA, dB, optimizer moments and master parameters are fp32.
+ *     dtype TEMPLORA_F32: everything is fp32.
+ *   - Data pointers must be 16-byte aligned.  The tensor-core path (bf16, d_in, d_out
+ *     and r multiples of 8, r <= 256) is taken automatically; other shapes run on a
+ *     generic kernel path.  r <= 256 always (the paper sweeps rank 16..256).
+ *   - Workspace: 256-byte aligned, at least templora_*workspace_bytes() long, and its
+ *     first 1024 bytes zeroed by the caller once before first use (they hold the
+ *     device status record).  A workspace must not be shared by calls that may
+ *     overlap on the GPU.
+ *   - Synchronous errors (bad argument, unsupported shape, short workspace, a CUDA
+ *     launch failure) are returned and nothing further is launched.  Device-side
+ *     problems (a bounded wait inside a kernel ran out) are recorded in the status
+ *     record at the head of the workspace; read it with templora_read_device_status.
+ */
+#ifndef TEMPLORA_H_
+#define TEMPLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TEMPLORA_OK = 0,
+  TEMPLORA_ERR_INVALID_ARG = 1,   /* NULL/misaligned pointer, non-positive size          */
+  TEMPLORA_ERR_UNSUPPORTED = 2,   /* shape or dtype outside what the kernels handle       */
+  TEMPLORA_ERR_WORKSPACE = 3,     /* workspace NULL, misaligned or too small              */
+  TEMPLORA_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                    */
+  TEMPLORA_ERR_TIMEOUT = 5        /* a bounded device-side wait expired (device status)   */
+} templora_status_t;
+
+typedef enum { TEMPLORA_F32 = 0, TEMPLORA_BF16 = 1 } templora_dtype_t;
+
+/* One LoRA-augmented projection (the temporary module attached to one frozen linear). */
+typedef struct {
+  int32_t d_in, d_out, r;
+  float s;            /* alpha / r                                                  */
+  int32_t dtype;      /* templora_dtype_t: storage type of x, W0, A, B, y, dY, dX   */
+  const void *W0;     /* [d_out, d_in]  frozen, read only                           */
+  const void *A;      /* [r, d_in]      working copy in `dtype`                     */
+  const void *B;      /* [d_out, r]     working copy in `dtype`                     */
+} templora_linear_t;
+
+/* Optimizer state of one tensor (an A or a B); all buffers caller-owned, n elements. */
+typedef struct {
+  int64_t n;
+  float *master;      /* fp32 parameter that AdamW updates                           */
+  float *m, *v;       /* fp32 first and second moments                               */
+  void *work;         /* copy in the working dtype re-emitted after each step
+                         (bf16, round-to-nearest-even); NULL when master is itself
+                         what the projections read (fp32 path)                       */
+  const float *grad;  /* fp32 gradient (dA or dB)                                    */
+} templora_param_t;
+
+/* Bytes of workspace sufficient for templora_linear_fwd, templora_linear_bwd and
+ * templora_decode_fwd on this projection with up to T rows.  0 on invalid input. */
+size_t templora_workspace_bytes(const templora_linear_t *lin, int32_t T);
+
+/* Bytes of workspace sufficient for templora_update_block on these projections. */
+size_t templora_update_block_workspace_bytes(const templora_linear_t *proj, int32_t n_proj, int32_t T);
+
+/*
+ * Forward of the LoRA-augmented projection over a chunk of T tokens
+ * (module forward inside "Train Theta_k", Algorithm 1; LoRA of the Section "Temp-Lora"):
+ *     U = x A^T ;  y = x W0^T + s U B^T
+ * x [T,d_in] in, y [T,d_out] out.  U_save: optional fp32 [T,r] that receives U
+ * (unscaled) for reuse by templora_linear_bwd; NULL to skip.
+ */
+templora_status_t templora_linear_fwd(const templora_linear_t *lin, int32_t T, const void *x, void *y,
+                                      float *U_save, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Backward of the same projection with W0 frozen (the method never alters the base
+ * model, so there is no dW0):
+ *     V = dY B ;  dX = dY W0 + s V A ;  dB = s dY^T U ;  dA = s V^T x
+ * U_saved: fp32 [T,r] from the forward, or NULL to recompute U = x A^T.
+ * dX [T,d_in] may be NULL (skipped).  dA [r,d_in], dB [d_out,r] are fp32 and are
+ * plain sums over the T tokens (no 1/T); accumulate != 0 adds to their contents.
+ */
+templora_status_t templora_linear_bwd(const templora_linear_t *lin, int32_t T, const void *x, const void *dY,
+                                      const float *U_saved, void *dX, float *dA, float *dB, int32_t accumulate,
+                                      void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * One AdamW step (decoupled weight decay, bias-corrected) on n_params tensors
+ * (optimizer step of "Train Theta_k"; learning rate 5e-5 in the paper's Setup,
+ * fp32 master weights and moments as bfloat16 ZeRO-2 training implies):
+ *     p <- p (1 - lr wd);  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2
+ *     p <- p - lr (m / (1-b1^step)) / (sqrt(v / (1-b2^step)) + eps)
+ * `step` is the 1-based index of this step.  params is a HOST array.
+ * If work_dtype is TEMPLORA_BF16 and work != NULL, work receives bf16(p).
+ */
+templora_status_t templora_adamw_step(const templora_param_t *params, int32_t n_params, float lr, float beta1,
+                                      float beta2, float eps, float weight_decay, int64_t step,
+                                      int32_t work_dtype, void *stream);
+
+/*
+ * Decode-time forward with the current (un-merged) module for n_tokens in 1..16 rows
+ * (generation step Y[i] = Theta_k(...) of Algorithm 1):  y = x W0^T + s (x A^T) B^T.
+ * Streams W0 once per call; bound by HBM bandwidth.
+ */
+templora_status_t templora_decode_fwd(const templora_linear_t *lin, int32_t n_tokens, const void *x, void *y,
+                                      void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The whole chunk update of n_proj projections: for each of `epochs` epochs, forward
+ * and backward of every projection over the T-token chunk with the current A, B, then
+ * one AdamW step on every A and B (batch = chunk, so one optimizer step per epoch;
+ * "n epochs" of Algorithm 1, n = 2 in the paper).
+ *   proj[i].A / .B must alias A_state[i].work / B_state[i].work (bf16) or .master (fp32);
+ *   gradients are written to A_state[i].grad / B_state[i].grad (cast away const inside:
+ *   the buffers are outputs of this call);
+ *   x[i] [T,d_in_i], dY[i] [T,d_out_i] inputs, constant across epochs;
+ *   y[i] [T,d_out_i] outputs (last epoch); dX[i] [T,d_in_i] outputs, dX or entries may be NULL.
+ *   *step_inout: number of optimizer steps already taken; incremented once per epoch.
+ * proj, A_state, B_state, x, dY, y, dX, step_inout are HOST memory.
+ */
+templora_status_t templora_update_block(const templora_linear_t *proj, const templora_param_t *A_state,
+                                        const templora_param_t *B_state, int32_t n_proj, int32_t T,
+                                        const void *const *x, const void *const *dY, void *const *y,
+                                        void *const *dX, int32_t epochs, float lr, float beta1, float beta2,
+                                        float eps, float weight_decay, int64_t *step_inout,
+                                        void *ws, size_t ws_bytes, void *stream);
+
+/* Static description of a status code. */
+const char *templora_status_string(templora_status_t st);
+
+/*
+ * Synchronises `stream`, then copies the device status record at the head of `ws`
+ * into *code (a templora_status_t; TEMPLORA_OK if no kernel reported a problem) and
+ * *where (an internal location tag).  Returns TEMPLORA_OK if the record was read.
+ */
+templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *code, int32_t *where);
+
+/*
+ * Kernel-path selection for testing: 0 = automatic (tensor-core path when the
+ * shape allows), 1 = always the generic kernel path.  Returns the previous value.
+ * Process-wide; not part of the method.
+ */
+int32_t templora_set_kernel_path(int32_t mode);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TEMPLORA_H_ */

@@ -1,0 +1,609 @@
+// C-ABI entry points: argument checks, workspace carving and the launch sequences of the
+// Temp-Lora chunk update (forward, backward, AdamW, epochs) and of the decode-time forward.
+#include "common.cuh"
+
+#include <atomic>
+#include <vector>
+
+namespace templora {
+namespace {
+
+std::atomic<int> g_kernel_path{0};      // 0 = automatic, 1 = generic kernels only
+thread_local int t_path_override = -1;  // set while measuring the workspace needs of both paths
+
+constexpr int kSmRef = 148;  // SM count the split-K heuristic is tuned for (B200)
+
+// Workspace bump allocator.  With base == nullptr it only measures.
+struct WsAlloc {
+  uint8_t *base;
+  size_t off, cap;
+  bool overflow = false;
+  WsAlloc(void *b, size_t c) : base(reinterpret_cast<uint8_t *>(b)), off(kStatusBytes), cap(c) {}
+  template <typename T> T *take(size_t count) {
+    size_t bytes = align_up(count * sizeof(T), kWsAlign);
+    size_t at = off;
+    off += bytes;
+    if (!base) return reinterpret_cast<T *>(uintptr_t(kWsAlign));  // dummy non-null
+    if (off > cap) { overflow = true; return nullptr; }
+    return reinterpret_cast<T *>(base + at);
+  }
+  DeviceStatus *status() const { return reinterpret_cast<DeviceStatus *>(base); }
+};
+
+inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// Split-K factor for a skinny problem: `tiles` output tiles, `kb` k-blocks of 64 each, launched
+// together with (group-1) similar problems.  Aims at about three work items per SM, never fewer
+// than 8 k-blocks per item, at most 16 splits.
+int pick_splits(int tiles, int kb, int group) {
+  long long total = (long long)tiles * kb * (group < 1 ? 1 : group);
+  long long target = (total + kSmRef * 3 - 1) / (kSmRef * 3);
+  if (target < 8) target = 8;
+  long long s = (kb + target / 2) / target;
+  if (s < 1) s = 1;
+  if (s > 16) s = 16;
+  if (s > kb) s = kb;
+  return (int)s;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+templora_status_t check_linear(const templora_linear_t *lin) {
+  if (!lin) return TEMPLORA_ERR_INVALID_ARG;
+  if (lin->d_in <= 0 || lin->d_out <= 0 || lin->r <= 0) return TEMPLORA_ERR_INVALID_ARG;
+  if (lin->dtype != TEMPLORA_F32 && lin->dtype != TEMPLORA_BF16) return TEMPLORA_ERR_UNSUPPORTED;
+  if (lin->r > 256) return TEMPLORA_ERR_UNSUPPORTED;
+  if (!(lin->s == lin->s)) return TEMPLORA_ERR_INVALID_ARG;
+  return TEMPLORA_OK;
+}
+templora_status_t check_linear_ptrs(const templora_linear_t *lin) {
+  if (!lin->W0 || !lin->A || !lin->B) return TEMPLORA_ERR_INVALID_ARG;
+  if (!aligned16(lin->W0) || !aligned16(lin->A) || !aligned16(lin->B)) return TEMPLORA_ERR_INVALID_ARG;
+  return TEMPLORA_OK;
+}
+templora_status_t check_ws(const void *ws, size_t ws_bytes) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < kStatusBytes) return TEMPLORA_ERR_WORKSPACE;
+  return TEMPLORA_OK;
+}
+
+// Does this projection take the tensor-core path?
+bool use_tc(const templora_linear_t *lin, bool dry) {
+  const int mode = t_path_override >= 0 ? t_path_override : g_kernel_path.load();
+  if (mode == 1) return false;
+  if (lin->dtype != TEMPLORA_BF16) return false;
+  if ((lin->d_in | lin->d_out | lin->r) & 7) return false;
+  return dry ? true : tc_available();
+}
+
+Operand op(const void *p, int dt, long long s0, long long s1) { return Operand{p, dt, s0, s1}; }
+
+// ---------------------------------------------------------------- problem builders (tensor-core path)
+TcProblem prob_U(const templora_linear_t *l, int T, const void *x, float *part, int splits) {
+  TcProblem p{};
+  p.M = T; p.N = l->r; p.K = l->d_in;
+  p.A = x; p.lda = l->d_in; p.a_mn = 0;
+  p.B = l->A; p.ldb = l->d_in; p.b_mn = 0;
+  p.splits = splits; p.out = part; p.out_f32 = 1; p.out_s0 = l->r; p.out_s1 = 1; p.out_split = (long long)T * l->r;
+  return p;
+}
+TcProblem prob_V(const templora_linear_t *l, int T, const void *dY, float *part, int splits) {
+  TcProblem p{};
+  p.M = T; p.N = l->r; p.K = l->d_out;
+  p.A = dY; p.lda = l->d_out; p.a_mn = 0;
+  p.B = l->B; p.ldb = l->r; p.b_mn = 1;   // B [d_out, r]: the contraction index d_out is the row index
+  p.splits = splits; p.out = part; p.out_f32 = 1; p.out_s0 = l->r; p.out_s1 = 1; p.out_split = (long long)T * l->r;
+  return p;
+}
+TcProblem prob_y(const templora_linear_t *l, int T, const void *x, const void *Us, void *y) {
+  TcProblem p{};
+  p.M = T; p.N = l->d_out; p.K = l->d_in; p.Kext = l->r;
+  p.A = x; p.lda = l->d_in; p.a_mn = 0;
+  p.B = l->W0; p.ldb = l->d_in; p.b_mn = 0;
+  p.Aext = Us; p.ldaext = l->r; p.Bext = l->B; p.ldbext = l->r;
+  p.splits = 1; p.out = y; p.out_f32 = 0; p.out_s0 = l->d_out; p.out_s1 = 1;
+  return p;
+}
+TcProblem prob_dX(const templora_linear_t *l, int T, const void *dY, const void *Vs, void *dX) {
+  TcProblem p{};
+  p.M = T; p.N = l->d_in; p.K = l->d_out; p.Kext = l->r;
+  p.A = dY; p.lda = l->d_out; p.a_mn = 0;
+  p.B = l->W0; p.ldb = l->d_in; p.b_mn = 1;    // W0 [d_out, d_in] contracted over its rows
+  p.Aext = Vs; p.ldaext = l->r; p.Bext = l->A; p.ldbext = l->d_in;  // A [r, d_in] contracted over its rows
+  p.splits = 1; p.out = dX; p.out_f32 = 0; p.out_s0 = l->d_in; p.out_s1 = 1;
+  return p;
+}
+TcProblem prob_dB(const templora_linear_t *l, int T, const void *dY, const void *Us, float *out, int splits) {
+  TcProblem p{};
+  p.M = l->d_out; p.N = l->r; p.K = T;
+  p.A = dY; p.lda = l->d_out; p.a_mn = 1;     // dY^T
+  p.B = Us; p.ldb = l->r; p.b_mn = 1;         // Us [T, r] holds s*U
+  p.splits = splits; p.out = out; p.out_f32 = 1; p.out_s0 = l->r; p.out_s1 = 1;
+  p.out_split = (long long)l->d_out * l->r;
+  return p;
+}
+TcProblem prob_dA(const templora_linear_t *l, int T, const void *x, const void *Vs, float *out, int splits) {
+  TcProblem p{};
+  p.M = l->d_in; p.N = l->r; p.K = T;         // computes dA^T = x^T (s V), stored transposed
+  p.A = x; p.lda = l->d_in; p.a_mn = 1;
+  p.B = Vs; p.ldb = l->r; p.b_mn = 1;
+  p.splits = splits; p.out = out; p.out_f32 = 1; p.out_s0 = 1; p.out_s1 = l->d_in;
+  p.out_split = (long long)l->d_in * l->r;
+  return p;
+}
+
+int splits_skinny(int T, int r, int K, int group) { return pick_splits(cdiv(T, 128) * cdiv(r, 64), cdiv(K, 64), group); }
+int splits_grad(int d, int r, int T, int group) { return pick_splits(cdiv(d, 128) * cdiv(r, 64), cdiv(T, 64), group); }
+
+// ---------------------------------------------------------------- forward
+templora_status_t fwd_impl(const templora_linear_t *l, int T, const void *x, void *y, float *U_save, WsAlloc &ws,
+                           bool dry, cudaStream_t st) {
+  const long long Tr = (long long)T * l->r;
+  if (use_tc(l, dry)) {
+    const int su = splits_skinny(T, l->r, l->d_in, 1);
+    float *Upart = ws.take<float>((size_t)su * Tr);
+    __nv_bfloat16 *Us = ws.take<__nv_bfloat16>((size_t)Tr);
+    if (dry) return TEMPLORA_OK;
+    if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+    TcProblem pu = prob_U(l, T, x, Upart, su);
+    TL_TRY(tc_gemm_grouped(&pu, 1, 64, ws.status(), st));
+    ReduceJob rj{Upart, su, Tr, Tr, l->s, 1.f, U_save, 0, Us};
+    TL_TRY(reduce_partials_batch(&rj, 1, st));
+    TcProblem py = prob_y(l, T, x, Us, y);
+    return tc_gemm_grouped(&py, 1, 256, ws.status(), st);
+  }
+  float *U = U_save ? U_save : ws.take<float>((size_t)Tr);
+  if (dry) return TEMPLORA_OK;
+  if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+  const int dt = l->dtype;
+  SimtGemm g{};
+  g.M = T; g.N = l->r; g.K1 = l->d_in; g.K2 = 0;
+  g.A1 = op(x, dt, l->d_in, 1); g.B1 = op(l->A, dt, 1, l->d_in);
+  g.alpha1 = 1.f; g.alpha2 = 0.f; g.D = U; g.d_dt = TEMPLORA_F32; g.ds0 = l->r; g.ds1 = 1;
+  TL_TRY(simt_gemm(g, st));
+  SimtGemm h{};
+  h.M = T; h.N = l->d_out; h.K1 = l->d_in; h.K2 = l->r;
+  h.A1 = op(x, dt, l->d_in, 1); h.B1 = op(l->W0, dt, 1, l->d_in);
+  h.A2 = op(U, TEMPLORA_F32, l->r, 1); h.B2 = op(l->B, dt, 1, l->r);
+  h.alpha1 = 1.f; h.alpha2 = l->s; h.D = y; h.d_dt = dt; h.ds0 = l->d_out; h.ds1 = 1;
+  return simt_gemm(h, st);
+}
+
+// ---------------------------------------------------------------- backward
+templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, const void *dY, const float *U_saved,
+                           void *dX, float *dA, float *dB, int accumulate, WsAlloc &ws, bool dry, cudaStream_t st) {
+  const long long Tr = (long long)T * l->r;
+  if (use_tc(l, dry)) {
+    const int su = U_saved ? 1 : splits_skinny(T, l->r, l->d_in, 2);
+    const int sv = splits_skinny(T, l->r, l->d_out, 2);
+    const int sb = splits_grad(l->d_out, l->r, T, 2), sa = splits_grad(l->d_in, l->r, T, 2);
+    float *Upart = U_saved ? nullptr : ws.take<float>((size_t)su * Tr);
+    float *Vpart = ws.take<float>((size_t)sv * Tr);
+    __nv_bfloat16 *Us = ws.take<__nv_bfloat16>((size_t)Tr);
+    __nv_bfloat16 *Vs = ws.take<__nv_bfloat16>((size_t)Tr);
+    const bool direct_b = (sb == 1 && !accumulate), direct_a = (sa == 1 && !accumulate);
+    float *dBpart = direct_b ? dB : ws.take<float>((size_t)sb * l->d_out * l->r);
+    float *dApart = direct_a ? dA : ws.take<float>((size_t)sa * l->d_in * l->r);
+    if (dry) return TEMPLORA_OK;
+    if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+
+    TcProblem skinny[2];
+    int ns = 0;
+    skinny[ns++] = prob_V(l, T, dY, Vpart, sv);
+    if (!U_saved) skinny[ns++] = prob_U(l, T, x, Upart, su);
+    TL_TRY(tc_gemm_grouped(skinny, ns, 64, ws.status(), st));
+    ReduceJob jobs[2] = {
+        ReduceJob{Vpart, sv, Tr, Tr, l->s, 1.f, nullptr, 0, Vs},
+        ReduceJob{U_saved ? U_saved : Upart, su, Tr, Tr, l->s, 1.f, nullptr, 0, Us},
+    };
+    TL_TRY(reduce_partials_batch(jobs, 2, st));
+    if (dX) {
+      TcProblem px = prob_dX(l, T, dY, Vs, dX);
+      TL_TRY(tc_gemm_grouped(&px, 1, 256, ws.status(), st));
+    }
+    TcProblem grads[2] = {prob_dB(l, T, dY, Us, dBpart, sb), prob_dA(l, T, x, Vs, dApart, sa)};
+    TL_TRY(tc_gemm_grouped(grads, 2, 64, ws.status(), st));
+    ReduceJob rj[2];
+    int nr = 0;
+    const long long nb = (long long)l->d_out * l->r, na = (long long)l->d_in * l->r;
+    if (!direct_b) rj[nr++] = ReduceJob{dBpart, sb, nb, nb, 1.f, 1.f, dB, accumulate, nullptr};
+    if (!direct_a) rj[nr++] = ReduceJob{dApart, sa, na, na, 1.f, 1.f, dA, accumulate, nullptr};
+    if (nr) TL_TRY(reduce_partials_batch(rj, nr, st));
+    return TEMPLORA_OK;
+  }
+  float *Ubuf = U_saved ? nullptr : ws.take<float>((size_t)Tr);
+  float *V = ws.take<float>((size_t)Tr);
+  if (dry) return TEMPLORA_OK;
+  if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+  const int dt = l->dtype;
+  const float *U = U_saved;
+  if (!U) {
+    SimtGemm g{};
+    g.M = T; g.N = l->r; g.K1 = l->d_in;
+    g.A1 = op(x, dt, l->d_in, 1); g.B1 = op(l->A, dt, 1, l->d_in);
+    g.alpha1 = 1.f; g.D = Ubuf; g.d_dt = TEMPLORA_F32; g.ds0 = l->r; g.ds1 = 1;
+    TL_TRY(simt_gemm(g, st));
+    U = Ubuf;
+  }
+  {  // V = dY B
+    SimtGemm g{};
+    g.M = T; g.N = l->r; g.K1 = l->d_out;
+    g.A1 = op(dY, dt, l->d_out, 1); g.B1 = op(l->B, dt, l->r, 1);
+    g.alpha1 = 1.f; g.D = V; g.d_dt = TEMPLORA_F32; g.ds0 = l->r; g.ds1 = 1;
+    TL_TRY(simt_gemm(g, st));
+  }
+  if (dX) {  // dX = dY W0 + s V A
+    SimtGemm g{};
+    g.M = T; g.N = l->d_in; g.K1 = l->d_out; g.K2 = l->r;
+    g.A1 = op(dY, dt, l->d_out, 1); g.B1 = op(l->W0, dt, l->d_in, 1);
+    g.A2 = op(V, TEMPLORA_F32, l->r, 1); g.B2 = op(l->A, dt, l->d_in, 1);
+    g.alpha1 = 1.f; g.alpha2 = l->s; g.D = dX; g.d_dt = dt; g.ds0 = l->d_in; g.ds1 = 1;
+    TL_TRY(simt_gemm(g, st));
+  }
+  {  // dB = s dY^T U
+    SimtGemm g{};
+    g.M = l->d_out; g.N = l->r; g.K1 = T;
+    g.A1 = op(dY, dt, 1, l->d_out); g.B1 = op(U, TEMPLORA_F32, l->r, 1);
+    g.alpha1 = l->s; g.D = dB; g.d_dt = TEMPLORA_F32; g.ds0 = l->r; g.ds1 = 1; g.accumulate = accumulate;
+    TL_TRY(simt_gemm(g, st));
+  }
+  {  // dA = s V^T x
+    SimtGemm g{};
+    g.M = l->r; g.N = l->d_in; g.K1 = T;
+    g.A1 = op(V, TEMPLORA_F32, 1, l->r); g.B1 = op(x, dt, l->d_in, 1);
+    g.alpha1 = l->s; g.D = dA; g.d_dt = TEMPLORA_F32; g.ds0 = l->d_in; g.ds1 = 1; g.accumulate = accumulate;
+    TL_TRY(simt_gemm(g, st));
+  }
+  return TEMPLORA_OK;
+}
+
+// ---------------------------------------------------------------- decode
+// y[i,o] = sum_k P[k][i][o] + s * sum_j (sum_k Pu[k][i][j]) * B[o][j]     (rank-r term added in registers)
+constexpr int kFinThreads = 128;
+__global__ void __launch_bounds__(kFinThreads) decode_finish_kernel(const float *__restrict__ P, int sp,
+                                                                    const float *__restrict__ Pu, int spu, int n,
+                                                                    int d_out, int r, float s,
+                                                                    const __nv_bfloat16 *__restrict__ B,
+                                                                    __nv_bfloat16 *__restrict__ y) {
+  extern __shared__ float u_sm[];  // [n][r], already scaled by s
+  for (int e = threadIdx.x; e < n * r; e += kFinThreads) {
+    float a = 0.f;
+    for (int k = 0; k < spu; ++k) a += Pu[(long long)k * n * r + e];
+    u_sm[e] = s * a;
+  }
+  __syncthreads();
+  const int o = blockIdx.x * kFinThreads + threadIdx.x;
+  if (o >= d_out) return;
+  float acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    acc[i] = 0.f;
+    if (i < n)
+      for (int k = 0; k < sp; ++k) acc[i] += P[((long long)k * n + i) * d_out + o];
+  }
+  const __nv_bfloat16 *brow = B + (long long)o * r;
+  for (int j0 = 0; j0 < r; j0 += 8) {  // r is a multiple of 8 on this path
+    uint4 w = *reinterpret_cast<const uint4 *>(brow + j0);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&w);
+    float b[8];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float2 f = __bfloat1622float2(h[e]);
+      b[2 * e] = f.x; b[2 * e + 1] = f.y;
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      if (i < n) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[i] = fmaf(u_sm[i * r + j0 + e], b[e], acc[i]);
+      }
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i)
+    if (i < n) y[(long long)i * d_out + o] = __float2bfloat16_rn(acc[i]);
+}
+
+templora_status_t decode_impl(const templora_linear_t *l, int n, const void *x, void *y, WsAlloc &ws, bool dry,
+                              cudaStream_t st) {
+  if (use_tc(l, dry)) {
+    const int kb = cdiv(l->d_in, 64);
+    const int sp = pick_splits(cdiv(l->d_out, 128), kb, 1);
+    const int spu = pick_splits(cdiv(l->r, 128), kb, 1);
+    float *P = ws.take<float>((size_t)sp * 16 * l->d_out);
+    float *Pu = ws.take<float>((size_t)spu * 16 * l->r);
+    if (dry) return TEMPLORA_OK;
+    if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+    TcProblem p[2] = {};
+    p[0].M = l->d_out; p[0].N = n; p[0].K = l->d_in;
+    p[0].A = l->W0; p[0].lda = l->d_in; p[0].B = x; p[0].ldb = l->d_in;
+    p[0].splits = sp; p[0].out = P; p[0].out_f32 = 1; p[0].out_s0 = 1; p[0].out_s1 = l->d_out;
+    p[0].out_split = (long long)n * l->d_out;
+    p[1].M = l->r; p[1].N = n; p[1].K = l->d_in;
+    p[1].A = l->A; p[1].lda = l->d_in; p[1].B = x; p[1].ldb = l->d_in;
+    p[1].splits = spu; p[1].out = Pu; p[1].out_f32 = 1; p[1].out_s0 = 1; p[1].out_s1 = l->r;
+    p[1].out_split = (long long)n * l->r;
+    TL_TRY(tc_gemm_grouped(p, 2, 16, ws.status(), st));
+    decode_finish_kernel<<<cdiv(l->d_out, kFinThreads), kFinThreads, (size_t)n * l->r * sizeof(float), st>>>(
+        P, sp, Pu, spu, n, l->d_out, l->r, l->s, reinterpret_cast<const __nv_bfloat16 *>(l->B),
+        reinterpret_cast<__nv_bfloat16 *>(y));
+    TL_CUDA_CHECK(cudaGetLastError());
+    return TEMPLORA_OK;
+  }
+  return fwd_impl(l, n, x, y, nullptr, ws, dry, st);
+}
+
+// ---------------------------------------------------------------- update_block (tensor-core, grouped)
+constexpr int kGroup = 8;  // projections per grouped launch (two problems each)
+
+struct GroupBufs {
+  float *Upart[kGroup], *Vpart[kGroup], *dBpart[kGroup], *dApart[kGroup];
+  __nv_bfloat16 *Us[kGroup], *Vs[kGroup];
+  int su[kGroup], sv[kGroup], sb[kGroup], sa[kGroup];
+};
+
+void carve_group(const templora_linear_t *proj, int n, int T, WsAlloc &ws, GroupBufs &b) {
+  for (int i = 0; i < n; ++i) {
+    const templora_linear_t *l = proj + i;
+    const long long Tr = (long long)T * l->r;
+    b.su[i] = splits_skinny(T, l->r, l->d_in, 2 * n);
+    b.sv[i] = splits_skinny(T, l->r, l->d_out, 2 * n);
+    b.sb[i] = splits_grad(l->d_out, l->r, T, 2 * n);
+    b.sa[i] = splits_grad(l->d_in, l->r, T, 2 * n);
+    b.Upart[i] = ws.take<float>((size_t)b.su[i] * Tr);
+    b.Vpart[i] = ws.take<float>((size_t)b.sv[i] * Tr);
+    b.Us[i] = ws.take<__nv_bfloat16>((size_t)Tr);
+    b.Vs[i] = ws.take<__nv_bfloat16>((size_t)Tr);
+    b.dBpart[i] = b.sb[i] > 1 ? ws.take<float>((size_t)b.sb[i] * l->d_out * l->r) : nullptr;
+    b.dApart[i] = b.sa[i] > 1 ? ws.take<float>((size_t)b.sa[i] * l->d_in * l->r) : nullptr;
+  }
+}
+
+templora_status_t update_group_tc(const templora_linear_t *proj, const templora_param_t *As, const templora_param_t *Bs,
+                                  int n, int T, const void *const *x, const void *const *dY, void *const *y,
+                                  void *const *dX, const GroupBufs &b, DeviceStatus *status, cudaStream_t st) {
+  TcProblem probs[2 * kGroup];
+  ReduceJob jobs[2 * kGroup];
+  int np = 0, nj = 0;
+  for (int i = 0; i < n; ++i) {
+    const long long Tr = (long long)T * proj[i].r;
+    probs[np++] = prob_U(proj + i, T, x[i], b.Upart[i], b.su[i]);
+    probs[np++] = prob_V(proj + i, T, dY[i], b.Vpart[i], b.sv[i]);
+    jobs[nj++] = ReduceJob{b.Upart[i], b.su[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Us[i]};
+    jobs[nj++] = ReduceJob{b.Vpart[i], b.sv[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Vs[i]};
+  }
+  TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
+  TL_TRY(reduce_partials_batch(jobs, nj, st));
+  np = 0;
+  for (int i = 0; i < n; ++i) {
+    probs[np++] = prob_y(proj + i, T, x[i], b.Us[i], y[i]);
+    if (dX && dX[i]) probs[np++] = prob_dX(proj + i, T, dY[i], b.Vs[i], dX[i]);
+  }
+  TL_TRY(tc_gemm_grouped(probs, np, 256, status, st));
+  np = 0; nj = 0;
+  for (int i = 0; i < n; ++i) {
+    const templora_linear_t *l = proj + i;
+    float *gB = const_cast<float *>(Bs[i].grad), *gA = const_cast<float *>(As[i].grad);
+    probs[np++] = prob_dB(l, T, dY[i], b.Us[i], b.sb[i] > 1 ? b.dBpart[i] : gB, b.sb[i]);
+    probs[np++] = prob_dA(l, T, x[i], b.Vs[i], b.sa[i] > 1 ? b.dApart[i] : gA, b.sa[i]);
+    const long long nb = (long long)l->d_out * l->r, na = (long long)l->d_in * l->r;
+    if (b.sb[i] > 1) jobs[nj++] = ReduceJob{b.dBpart[i], b.sb[i], nb, nb, 1.f, 1.f, gB, 0, nullptr};
+    if (b.sa[i] > 1) jobs[nj++] = ReduceJob{b.dApart[i], b.sa[i], na, na, 1.f, 1.f, gA, 0, nullptr};
+  }
+  TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
+  if (nj) TL_TRY(reduce_partials_batch(jobs, nj, st));
+  return TEMPLORA_OK;
+}
+
+templora_status_t update_impl(const templora_linear_t *proj, const templora_param_t *As, const templora_param_t *Bs,
+                              int n_proj, int T, const void *const *x, const void *const *dY, void *const *y,
+                              void *const *dX, int epochs, float lr, float b1, float b2, float eps, float wd,
+                              int64_t *step_inout, void *ws_ptr, size_t ws_bytes, bool dry, size_t *need,
+                              cudaStream_t st) {
+  bool all_tc = true;
+  for (int i = 0; i < n_proj; ++i) all_tc = all_tc && use_tc(proj + i, dry);
+  // workspace: the largest need of any group (groups run one after another on the stream)
+  size_t max_need = kStatusBytes;
+  if (all_tc) {
+    for (int g0 = 0; g0 < n_proj; g0 += kGroup) {
+      WsAlloc m(nullptr, 0);
+      GroupBufs gb;
+      carve_group(proj + g0, (n_proj - g0 < kGroup) ? n_proj - g0 : kGroup, T, m, gb);
+      if (m.off > max_need) max_need = m.off;
+    }
+  } else {
+    for (int i = 0; i < n_proj; ++i) {
+      WsAlloc m(nullptr, 0);
+      fwd_impl(proj + i, T, nullptr, nullptr, nullptr, m, true, st);
+      if (m.off > max_need) max_need = m.off;
+      WsAlloc m2(nullptr, 0);
+      bwd_impl(proj + i, T, nullptr, nullptr, nullptr, reinterpret_cast<void *>(16), nullptr, nullptr, 0, m2, true, st);
+      if (m2.off > max_need) max_need = m2.off;
+    }
+  }
+  if (need) *need = max_need;
+  if (dry) return TEMPLORA_OK;
+  if (ws_bytes < max_need) return TEMPLORA_ERR_WORKSPACE;
+
+  std::vector<templora_param_t> all;
+  all.reserve(2 * (size_t)n_proj);
+  for (int i = 0; i < n_proj; ++i) { all.push_back(As[i]); all.push_back(Bs[i]); }
+  const int work_bf16 = proj[0].dtype == TEMPLORA_BF16;
+  int64_t step = *step_inout;
+  for (int e = 0; e < epochs; ++e) {
+    if (all_tc) {
+      for (int g0 = 0; g0 < n_proj; g0 += kGroup) {
+        const int n = (n_proj - g0 < kGroup) ? n_proj - g0 : kGroup;
+        WsAlloc a(ws_ptr, ws_bytes);
+        GroupBufs gb;
+        carve_group(proj + g0, n, T, a, gb);
+        if (a.overflow) return TEMPLORA_ERR_WORKSPACE;
+        TL_TRY(update_group_tc(proj + g0, As + g0, Bs + g0, n, T, x + g0, dY + g0, y + g0, dX ? dX + g0 : nullptr, gb,
+                               a.status(), st));
+      }
+    } else {
+      for (int i = 0; i < n_proj; ++i) {
+        WsAlloc a(ws_ptr, ws_bytes);
+        TL_TRY(fwd_impl(proj + i, T, x[i], y[i], nullptr, a, false, st));
+        WsAlloc c(ws_ptr, ws_bytes);
+        TL_TRY(bwd_impl(proj + i, T, x[i], dY[i], nullptr, dX ? dX[i] : nullptr, const_cast<float *>(As[i].grad),
+                        const_cast<float *>(Bs[i].grad), 0, c, false, st));
+      }
+    }
+    ++step;
+    TL_TRY(adamw_launch(all.data(), (int)all.size(), lr, b1, b2, eps, wd, step, work_bf16, st));
+    *step_inout = step;
+  }
+  return TEMPLORA_OK;
+}
+
+}  // namespace
+}  // namespace templora
+
+using namespace templora;
+
+extern "C" {
+
+size_t templora_workspace_bytes(const templora_linear_t *lin, int32_t T) {
+  if (check_linear(lin) != TEMPLORA_OK || T <= 0) return 0;
+  size_t need = kStatusBytes;
+  cudaStream_t st = nullptr;
+  // measure both kernel paths so that the figure holds whichever is selected later
+  for (int mode = 0; mode < 2; ++mode) {
+    t_path_override = mode;
+    WsAlloc a(nullptr, 0);
+    fwd_impl(lin, T, nullptr, nullptr, nullptr, a, true, st);
+    if (a.off > need) need = a.off;
+    WsAlloc b(nullptr, 0);
+    bwd_impl(lin, T, nullptr, nullptr, nullptr, reinterpret_cast<void *>(16), nullptr, nullptr, 1, b, true, st);
+    if (b.off > need) need = b.off;
+    WsAlloc c(nullptr, 0);
+    decode_impl(lin, T < 16 ? T : 16, nullptr, nullptr, c, true, st);
+    if (c.off > need) need = c.off;
+  }
+  t_path_override = -1;
+  return need;
+}
+
+size_t templora_update_block_workspace_bytes(const templora_linear_t *proj, int32_t n_proj, int32_t T) {
+  if (!proj || n_proj <= 0 || T <= 0) return 0;
+  for (int i = 0; i < n_proj; ++i)
+    if (check_linear(proj + i) != TEMPLORA_OK) return 0;
+  size_t need = 0, best = kStatusBytes;
+  for (int mode = 0; mode < 2; ++mode) {
+    t_path_override = mode;
+    update_impl(proj, nullptr, nullptr, n_proj, T, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0, 0, nullptr, nullptr,
+                0, true, &need, nullptr);
+    if (need > best) best = need;
+  }
+  t_path_override = -1;
+  return best;
+}
+
+templora_status_t templora_linear_fwd(const templora_linear_t *lin, int32_t T, const void *x, void *y, float *U_save,
+                                      void *ws, size_t ws_bytes, void *stream) {
+  TL_TRY(check_linear(lin));
+  TL_TRY(check_linear_ptrs(lin));
+  if (T <= 0 || !x || !y || !aligned16(x) || !aligned16(y) || (U_save && !aligned16(U_save))) return TEMPLORA_ERR_INVALID_ARG;
+  TL_TRY(check_ws(ws, ws_bytes));
+  WsAlloc a(ws, ws_bytes);
+  return fwd_impl(lin, T, x, y, U_save, a, false, reinterpret_cast<cudaStream_t>(stream));
+}
+
+templora_status_t templora_linear_bwd(const templora_linear_t *lin, int32_t T, const void *x, const void *dY,
+                                      const float *U_saved, void *dX, float *dA, float *dB, int32_t accumulate,
+                                      void *ws, size_t ws_bytes, void *stream) {
+  TL_TRY(check_linear(lin));
+  TL_TRY(check_linear_ptrs(lin));
+  if (T <= 0 || !x || !dY || !dA || !dB) return TEMPLORA_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(dY) || !aligned16(dA) || !aligned16(dB) || (dX && !aligned16(dX)) ||
+      (U_saved && !aligned16(U_saved)))
+    return TEMPLORA_ERR_INVALID_ARG;
+  TL_TRY(check_ws(ws, ws_bytes));
+  WsAlloc a(ws, ws_bytes);
+  return bwd_impl(lin, T, x, dY, U_saved, dX, dA, dB, accumulate ? 1 : 0, a, false, reinterpret_cast<cudaStream_t>(stream));
+}
+
+templora_status_t templora_adamw_step(const templora_param_t *params, int32_t n_params, float lr, float beta1,
+                                      float beta2, float eps, float weight_decay, int64_t step, int32_t work_dtype,
+                                      void *stream) {
+  if (!params || n_params <= 0 || step < 1) return TEMPLORA_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f) || !(lr == lr)) return TEMPLORA_ERR_INVALID_ARG;
+  if (work_dtype != TEMPLORA_F32 && work_dtype != TEMPLORA_BF16) return TEMPLORA_ERR_UNSUPPORTED;
+  for (int i = 0; i < n_params; ++i) {
+    const templora_param_t &p = params[i];
+    if (p.n <= 0 || !p.master || !p.m || !p.v || !p.grad) return TEMPLORA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(p.master) | reinterpret_cast<uintptr_t>(p.m) | reinterpret_cast<uintptr_t>(p.v) |
+         reinterpret_cast<uintptr_t>(p.grad)) & 3)
+      return TEMPLORA_ERR_INVALID_ARG;
+  }
+  return adamw_launch(params, n_params, lr, beta1, beta2, eps, weight_decay, step, work_dtype == TEMPLORA_BF16,
+                      reinterpret_cast<cudaStream_t>(stream));
+}
+
+templora_status_t templora_decode_fwd(const templora_linear_t *lin, int32_t n_tokens, const void *x, void *y, void *ws,
+                                      size_t ws_bytes, void *stream) {
+  TL_TRY(check_linear(lin));
+  TL_TRY(check_linear_ptrs(lin));
+  if (n_tokens < 1 || n_tokens > 16) return TEMPLORA_ERR_INVALID_ARG;
+  if (!x || !y || !aligned16(x) || !aligned16(y)) return TEMPLORA_ERR_INVALID_ARG;
+  TL_TRY(check_ws(ws, ws_bytes));
+  WsAlloc a(ws, ws_bytes);
+  return decode_impl(lin, n_tokens, x, y, a, false, reinterpret_cast<cudaStream_t>(stream));
+}
+
+templora_status_t templora_update_block(const templora_linear_t *proj, const templora_param_t *A_state,
+                                        const templora_param_t *B_state, int32_t n_proj, int32_t T,
+                                        const void *const *x, const void *const *dY, void *const *y, void *const *dX,
+                                        int32_t epochs, float lr, float beta1, float beta2, float eps,
+                                        float weight_decay, int64_t *step_inout, void *ws, size_t ws_bytes,
+                                        void *stream) {
+  if (!proj || !A_state || !B_state || n_proj <= 0 || T <= 0 || !x || !dY || !y || epochs < 0 || !step_inout ||
+      *step_inout < 0)
+    return TEMPLORA_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f)) return TEMPLORA_ERR_INVALID_ARG;
+  for (int i = 0; i < n_proj; ++i) {
+    TL_TRY(check_linear(proj + i));
+    TL_TRY(check_linear_ptrs(proj + i));
+    if (proj[i].dtype != proj[0].dtype) return TEMPLORA_ERR_UNSUPPORTED;
+    if (!x[i] || !dY[i] || !y[i] || !aligned16(x[i]) || !aligned16(dY[i]) || !aligned16(y[i])) return TEMPLORA_ERR_INVALID_ARG;
+    if (dX && dX[i] && !aligned16(dX[i])) return TEMPLORA_ERR_INVALID_ARG;
+    const templora_param_t &a = A_state[i], &b = B_state[i];
+    if (a.n != (int64_t)proj[i].r * proj[i].d_in || b.n != (int64_t)proj[i].d_out * proj[i].r) return TEMPLORA_ERR_INVALID_ARG;
+    if (!a.master || !a.m || !a.v || !a.grad || !b.master || !b.m || !b.v || !b.grad) return TEMPLORA_ERR_INVALID_ARG;
+    if (!aligned16(a.grad) || !aligned16(b.grad)) return TEMPLORA_ERR_INVALID_ARG;
+    // the projections must read what the optimizer writes
+    const void *wa = proj[i].dtype == TEMPLORA_BF16 ? a.work : (const void *)a.master;
+    const void *wb = proj[i].dtype == TEMPLORA_BF16 ? b.work : (const void *)b.master;
+    if (proj[i].A != wa || proj[i].B != wb) return TEMPLORA_ERR_INVALID_ARG;
+  }
+  TL_TRY(check_ws(ws, ws_bytes));
+  return update_impl(proj, A_state, B_state, n_proj, T, x, dY, y, dX, epochs, lr, beta1, beta2, eps, weight_decay,
+                     step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream));
+}
+
+const char *templora_status_string(templora_status_t st) {
+  switch (st) {
+    case TEMPLORA_OK: return "ok";
+    case TEMPLORA_ERR_INVALID_ARG: return "invalid argument";
+    case TEMPLORA_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case TEMPLORA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case TEMPLORA_ERR_CUDA: return "CUDA call failed";
+    case TEMPLORA_ERR_TIMEOUT: return "bounded device-side wait expired";
+  }
+  return "unknown status";
+}
+
+templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *code, int32_t *where) {
+  if (!ws || !code || !where) return TEMPLORA_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return TEMPLORA_ERR_CUDA;
+  int32_t rec[2] = {0, 0};
+  if (cudaMemcpy(rec, ws, sizeof(rec), cudaMemcpyDeviceToHost) != cudaSuccess) return TEMPLORA_ERR_CUDA;
+  *code = rec[0];
+  *where = rec[1];
+  return TEMPLORA_OK;
+}
+
+int32_t templora_set_kernel_path(int32_t mode) {
+  return g_kernel_path.exchange(mode == 1 ? 1 : 0);
+}
+
+}  // extern "C"

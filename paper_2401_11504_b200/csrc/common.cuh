@@ -1,0 +1,97 @@
+// Shared declarations of the Temp-Lora CUDA library (internal; the public ABI is include/templora.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "templora.h"
+
+namespace templora {
+
+// ---- device status record at the head of every workspace -------------------
+// code: templora_status_t (0 = ok); where: location tag of the first failure.
+struct DeviceStatus {
+  int32_t code;
+  int32_t where;
+  int32_t pad[62];
+};
+static_assert(sizeof(DeviceStatus) == 256, "status record is 256 bytes");
+
+constexpr size_t kWsAlign = 1024;
+constexpr size_t kStatusBytes = 1024;  // status record + padding; scratch starts here
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+#define TL_CUDA_CHECK(expr)                                   \
+  do {                                                        \
+    cudaError_t _e = (expr);                                  \
+    if (_e != cudaSuccess) return TEMPLORA_ERR_CUDA;          \
+  } while (0)
+
+#define TL_TRY(expr)                                          \
+  do {                                                        \
+    templora_status_t _s = (expr);                            \
+    if (_s != TEMPLORA_OK) return _s;                         \
+  } while (0)
+
+// ---- generic (SIMT) GEMM:  D = alpha1 * A1 B1 + alpha2 * A2 B2 (+ D) --------
+// Element (i,k) of an operand lives at p[i*s0 + k*s1]; dt is a templora_dtype_t.
+struct Operand {
+  const void *p;
+  int32_t dt;
+  long long s0, s1;
+};
+struct SimtGemm {
+  int M, N, K1, K2;          // K2 = 0: no second product
+  Operand A1, B1, A2, B2;    // A(i,k), B(k,j)
+  float alpha1, alpha2;
+  void *D;
+  int32_t d_dt;
+  long long ds0, ds1;
+  int accumulate;            // add to existing D (fp32 outputs only)
+};
+templora_status_t simt_gemm(const SimtGemm &g, cudaStream_t st);
+
+// ---- elementwise helpers ----------------------------------------------------
+// One reduction of split-K partial slabs, summed in slab order (deterministic):
+//   acc[i]      = sum_k part[k*stride + i]
+//   out_f32[i]  = scale_f32  * acc[i]  (+ previous contents when accumulate_f32)   if out_f32
+//   out_bf16[i] = bf16(scale_bf16 * acc[i])                                        if out_bf16
+struct ReduceJob {
+  const float *part;
+  int n_parts;
+  long long stride, n;
+  float scale_bf16;
+  float scale_f32;
+  float *out_f32;
+  int accumulate_f32;
+  __nv_bfloat16 *out_bf16;
+};
+templora_status_t reduce_partials_batch(const ReduceJob *jobs, int n_jobs, cudaStream_t st);
+
+// ---- AdamW --------------------------------------------------------------------
+templora_status_t adamw_launch(const templora_param_t *params, int n_params, float lr, float beta1, float beta2,
+                               float eps, float wd, int64_t step, int work_bf16, cudaStream_t st);
+
+// ---- tensor-core (tcgen05) grouped GEMM ---------------------------------------
+// D[M,N] = Aop[M,K] Bop[N,K]^T  (+ Aext[M,Kext] Bext[N,Kext]^T), bf16 operands, fp32 accumulation.
+// *_mn = 0: operand stored with K contiguous (rows = M or N, pitch ld elements)
+// *_mn = 1: operand stored with M (or N) contiguous (rows = K, pitch ld elements)
+struct TcProblem {
+  int M, N, K, Kext;
+  const void *A, *B, *Aext, *Bext;
+  long long lda, ldb, ldaext, ldbext;
+  int a_mn, b_mn;
+  int splits;                 // split-K factor (>= 1); split i writes out + i*out_split
+  void *out;
+  int out_f32;                // 1: fp32 output, 0: bf16
+  long long out_s0, out_s1;   // element (i,j) of D goes to out[i*out_s0 + j*out_s1]
+  long long out_split;        // element stride between split-K partial outputs
+};
+constexpr int kTcMaxProblems = 16;
+// BN: tile width, one of 16, 64, 256.
+templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st);
+bool tc_available();
+
+}  // namespace templora

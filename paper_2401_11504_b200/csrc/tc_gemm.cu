@@ -1,0 +1,536 @@
+// Persistent grouped GEMM on the sm_100a tensor cores (tcgen05 + TMEM accumulators, operands
+// staged by TMA).  One launch runs a list of problems
+//     D[M,N] = Aop[M,K] Bop[N,K]^T  (+ Aext[M,Kext] Bext[N,Kext]^T)
+// with bf16 operands and fp32 accumulation.  The optional second product runs as extra
+// k-blocks of the same tile loop into the same TMEM accumulator: that is how the rank-r LoRA
+// term s U B^T (forward) and s V A (input gradient) are fused into the frozen-weight GEMM.
+// Either operand may be stored K-contiguous or M/N-contiguous, so dY W0 (W0 row-major, contracted
+// over its rows) and the token-dimension reductions dY^T U and x^T V need no transposed copies.
+// Split-K partial outputs are written to separate slabs and summed later in a fixed order.
+//
+// CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns TMEM and issues the MMAs, warps 2..5 drain
+// the accumulator (TMEM -> registers -> global).  Two accumulator buffers let the epilogue of one
+// tile overlap the mainloop of the next.  Every mbarrier wait is bounded: when a wait runs out the
+// CTA records TEMPLORA_ERR_TIMEOUT in the device status record, drains what it has in flight,
+// frees its TMEM and returns.
+#include "common.cuh"
+
+#include <cuda.h>
+
+namespace templora {
+namespace {
+
+constexpr int BM = 128, BK = 64;
+constexpr int kThreads = 192;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+constexpr int kStageA = BM * BK * 2;  // 16 KB
+template <int BN, int STAGES, int TMEM_COLS> struct CfgBase {
+  static constexpr int kStages = STAGES, kTmemCols = TMEM_COLS;
+  static constexpr int kStageB = BN * BK * 2;
+  static constexpr int kStage = kStageA + kStageB;
+  static constexpr int kSmemBytes = STAGES * kStage + 1024 /*barriers*/ + 1024 /*alignment slack*/;
+};
+template <int BN> struct Cfg;
+template <> struct Cfg<256> : CfgBase<256, 4, 512> {};
+template <> struct Cfg<64> : CfgBase<64, 8, 128> {};
+template <> struct Cfg<16> : CfgBase<16, 10, 32> {};
+
+struct alignas(64) DevProb {
+  CUtensorMap tmA, tmB, tmAe, tmBe;
+  long long out_s0, out_s1, out_split;
+  void *out;
+  int M, N, kb_main, kb_ext, splits, m_tiles, n_tiles, item_start, a_mn, b_mn, out_f32, pad;
+};
+struct DevGroup {
+  DevProb p[kTcMaxProblems];
+  DeviceStatus *status;
+  int n_prob, n_items;
+};
+
+struct Item {
+  int p, m0, nt, split, kb0, kb1, next;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting or the limit ran out (then it also
+// raises the CTA's abort flag and records the location in the device status record).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, DeviceStatus *st,
+                                       int where) {
+  for (int i = 0; i < 4096; ++i)
+    if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  while (true) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      if (st && atomicCAS(&st->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) st->where = where;
+      __threadfence();
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version for tcgen05
+  d |= 2ull << 61;  // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(int n, int a_mn, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ Item decode_item(const DevGroup &g, int item) {
+  int p = 0;
+  while (p + 1 < g.n_prob && item >= g.p[p + 1].item_start) ++p;
+  const DevProb &q = g.p[p];
+  int local = item - q.item_start;
+  Item it;
+  it.p = p;
+  it.m0 = (local % q.m_tiles) * BM;
+  local /= q.m_tiles;
+  it.nt = local % q.n_tiles;
+  it.split = local / q.n_tiles;
+  it.kb0 = (int)((long long)q.kb_main * it.split / q.splits);
+  it.kb1 = (int)((long long)q.kb_main * (it.split + 1) / q.splits);
+  it.next = (it.split == q.splits - 1) ? q.kb_ext : 0;
+  return it;
+}
+
+// ------------------------------------------------------------------ epilogue stores
+template <int NV>
+__device__ __forceinline__ void store_chunk(const DevProb &q, const uint32_t (&v)[32], int row, int col0, int split) {
+  if (row >= q.M || col0 >= q.N) return;
+  const long long base = (long long)split * q.out_split + (long long)row * q.out_s0 + (long long)col0 * q.out_s1;
+  const int ncol = (q.N - col0 < NV) ? q.N - col0 : NV;
+  if (q.out_f32) {
+    float *o = reinterpret_cast<float *>(q.out) + base;
+    if (q.out_s1 == 1 && ncol == NV && ((reinterpret_cast<uintptr_t>(o) & 15) == 0)) {
+#pragma unroll
+      for (int c = 0; c < NV; c += 4)
+        *reinterpret_cast<float4 *>(o + c) = make_float4(__uint_as_float(v[c]), __uint_as_float(v[c + 1]),
+                                                         __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+    } else {
+#pragma unroll
+      for (int c = 0; c < NV; ++c)
+        if (c < ncol) o[(long long)c * q.out_s1] = __uint_as_float(v[c]);
+    }
+  } else {
+    __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(q.out) + base;
+    if (q.out_s1 == 1 && ncol == NV && ((reinterpret_cast<uintptr_t>(o) & 15) == 0)) {
+#pragma unroll
+      for (int c = 0; c < NV; c += 8) {
+        uint4 w;
+        __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(v[c]), __uint_as_float(v[c + 1]));
+        __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+        __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[c + 4]), __uint_as_float(v[c + 5]));
+        __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(v[c + 6]), __uint_as_float(v[c + 7]));
+        w.x = *reinterpret_cast<uint32_t *>(&t0);
+        w.y = *reinterpret_cast<uint32_t *>(&t1);
+        w.z = *reinterpret_cast<uint32_t *>(&t2);
+        w.w = *reinterpret_cast<uint32_t *>(&t3);
+        *reinterpret_cast<uint4 *>(o + c) = w;
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < NV; ++c)
+        if (c < ncol) o[(long long)c * q.out_s1] = __float2bfloat16_rn(__uint_as_float(v[c]));
+    }
+  }
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ DevGroup g) {
+  constexpr int kStages = Cfg<BN>::kStages;
+  constexpr int kStage = Cfg<BN>::kStage;
+  constexpr uint32_t kTxBytes = (uint32_t)kStage;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_al = smem_raw + (smem0 - smem_u32(smem_raw));
+  const uint32_t bar0 = smem0 + kStages * kStage;  // barriers: 8 bytes each
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + kStages * kStage + 512);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 516);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);
+    }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
+                 "r"((uint32_t)Cfg<BN>::kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      long long issued = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < g.n_items; item += gridDim.x) {
+        const Item it = decode_item(g, item);
+        const DevProb &q = g.p[it.p];
+        const int n0 = it.nt * BN;
+        const int nmain = it.kb1 - it.kb0;
+        const int nkb = nmain + it.next;
+        for (int i = 0; i < nkb; ++i) {
+          const bool ext = i >= nmain;
+          const int kel = ext ? (i - nmain) * BK : (it.kb0 + i) * BK;
+          const CUtensorMap *ma = ext ? &q.tmAe : &q.tmA;
+          const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 100)) { ok = false; break; }
+          mbar_arrive_expect_tx(full_bar(stage), kTxBytes);
+          const uint32_t sA = smem0 + stage * kStage, sB = sA + kStageA;
+          if (!q.a_mn) {
+            tma_load_2d(sA, ma, full_bar(stage), kel, it.m0);
+          } else {
+#pragma unroll
+            for (int b = 0; b < BM / 64; ++b) tma_load_2d(sA + b * 8192, ma, full_bar(stage), it.m0 + b * 64, kel);
+          }
+          if (!q.b_mn) {
+            tma_load_2d(sB, mb, full_bar(stage), kel, n0);
+          } else {
+#pragma unroll
+            for (int b = 0; b < (BN >= 64 ? BN / 64 : 1); ++b)
+              tma_load_2d(sB + b * 8192, mb, full_bar(stage), n0 + b * 64, kel);
+          }
+          ++issued;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // wait (bounded) for the copies this thread still has in flight before the CTA may exit
+        long long n = issued < kStages ? issued : kStages;
+        for (long long k = 0; k < n; ++k) {
+          long long idx = issued - 1 - k;
+          int s = (int)(idx % kStages);
+          uint32_t ph = (uint32_t)((idx / kStages) & 1);
+          const unsigned long long t0 = globaltimer_ns();
+          while (!mbar_try(full_bar(s), ph) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < g.n_items; item += gridDim.x, ++local) {
+        const Item it = decode_item(g, item);
+        const DevProb &q = g.p[it.p];
+        const int nkb = (it.kb1 - it.kb0) + it.next;
+        const int acc = local & 1;
+        const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, g.status, 200)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        const uint32_t idesc = instr_desc(BN, q.a_mn, q.b_mn);
+        for (int i = 0; i < nkb; ++i) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, g.status, 201)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sA = smem0 + stage * kStage, sB = sA + kStageA;
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            const uint64_t ad = q.a_mn ? smem_desc(sA + kk * 2048, 8192, 1024) : smem_desc(sA + kk * 32, 16, 1024);
+            const uint64_t bd = q.b_mn ? smem_desc(sB + kk * 2048, 8192, 1024) : smem_desc(sB + kk * 32, 16, 1024);
+            tc_mma_bf16(d_tmem, ad, bd, idesc, (i | kk) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));  // frees the smem stage once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit(tfull_bar(acc));  // accumulator complete
+      }
+      if (!ok) {
+        // let MMAs already issued finish before TMEM is released
+        tc_commit(drain_bar);
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try(drain_bar, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ===================== epilogue (warps 2..5) =====================
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
+    int local = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; ok && item < g.n_items; item += gridDim.x, ++local) {
+      const Item it = decode_item(g, item);
+      const DevProb &q = g.p[it.p];
+      const int n0 = it.nt * BN;
+      const int acc = local & 1;
+      const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, g.status, 300)) { ok = false; break; }
+      tc_fence_after();
+      const int row = it.m0 + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      uint32_t v[32];
+      if constexpr (BN >= 32) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld32(t_row + c0, v);
+          tmem_ld_wait();
+          store_chunk<32>(q, v, row, n0 + c0, it.split);
+        }
+      } else {
+        tmem_ld16(t_row, v);
+        tmem_ld_wait();
+        store_chunk<16>(q, v, row, n0, it.split);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg<BN>::kTmemCols)
+                 : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
+    if (qres != cudaDriverEntryPointSuccess) return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// 2-D bf16 tensor [outer][inner] with row pitch `pitch` elements; box = 64 x box_outer, 128B swizzle.
+bool make_map(CUtensorMap *m, const void *ptr, long long inner, long long outer, long long pitch, int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t gstr[1] = {(cuuint64_t)pitch * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// operand [rows = M or N][K] (mn = 0) or [K][M or N] (mn = 1)
+bool make_operand_map(CUtensorMap *m, const void *ptr, long long mn_extent, long long k_extent, long long ld, int mn,
+                      int tile_mn) {
+  if (!mn) return make_map(m, ptr, k_extent, mn_extent, ld, tile_mn);
+  return make_map(m, ptr, mn_extent, k_extent, ld, 64);
+}
+
+struct DeviceInfo {
+  int sm_count = 0;
+  int cc_major = 0;
+  bool attr_set[3] = {false, false, false};
+};
+DeviceInfo *device_info() {
+  static DeviceInfo info[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  DeviceInfo &d = info[dev];
+  if (d.sm_count == 0) {
+    int sm = 0, major = 0;
+    if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return nullptr;
+    d.cc_major = major;
+    d.sm_count = sm;
+  }
+  return &d;
+}
+
+template <int BN>
+templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream_t st) {
+  if (!di->attr_set[slot]) {
+    TL_CUDA_CHECK(cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes));
+    di->attr_set[slot] = true;
+  }
+  int grid = g.n_items < di->sm_count ? g.n_items : di->sm_count;
+  tc_gemm_kernel<BN><<<grid, kThreads, Cfg<BN>::kSmemBytes, st>>>(g);
+  TL_CUDA_CHECK(cudaGetLastError());
+  return TEMPLORA_OK;
+}
+
+}  // namespace
+
+bool tc_available() {
+  DeviceInfo *di = device_info();
+  return di && di->cc_major == 10 && encode_fn() != nullptr;
+}
+
+templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st) {
+  if (n <= 0 || n > kTcMaxProblems) return TEMPLORA_ERR_INVALID_ARG;
+  if (BN != 16 && BN != 64 && BN != 256) return TEMPLORA_ERR_INVALID_ARG;
+  DeviceInfo *di = device_info();
+  if (!di || di->cc_major != 10) return TEMPLORA_ERR_UNSUPPORTED;
+
+  // heaviest work items first: the static round-robin schedule then ends on the short ones
+  int order[kTcMaxProblems];
+  for (int i = 0; i < n; ++i) order[i] = i;
+  auto weight = [&](int i) {
+    const TcProblem &p = probs[i];
+    long long kb = (p.K + BK - 1) / BK;
+    int s = p.splits < 1 ? 1 : p.splits;
+    return (kb + s - 1) / s + (p.Kext + BK - 1) / BK;
+  };
+  for (int i = 1; i < n; ++i)
+    for (int j = i; j > 0 && weight(order[j]) > weight(order[j - 1]); --j) {
+      int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
+    }
+
+  DevGroup g;
+  g.status = status;
+  g.n_prob = n;
+  int items = 0;
+  for (int i = 0; i < n; ++i) {
+    const TcProblem &p = probs[order[i]];
+    DevProb &q = g.p[i];
+    if (p.M <= 0 || p.N <= 0 || p.K <= 0 || p.Kext < 0 || !p.A || !p.B || !p.out) return TEMPLORA_ERR_INVALID_ARG;
+    if (p.b_mn && BN < 64) return TEMPLORA_ERR_UNSUPPORTED;
+    if ((p.lda | p.ldb) & 7) return TEMPLORA_ERR_UNSUPPORTED;
+    q.M = p.M; q.N = p.N;
+    q.kb_main = (p.K + BK - 1) / BK;
+    q.kb_ext = (p.Kext + BK - 1) / BK;
+    q.splits = p.splits < 1 ? 1 : (p.splits > q.kb_main ? q.kb_main : p.splits);
+    q.m_tiles = (p.M + BM - 1) / BM;
+    q.n_tiles = (p.N + BN - 1) / BN;
+    q.item_start = items;
+    q.a_mn = p.a_mn; q.b_mn = p.b_mn;
+    q.out_f32 = p.out_f32; q.pad = 0;
+    q.out = p.out; q.out_s0 = p.out_s0; q.out_s1 = p.out_s1; q.out_split = p.out_split;
+    long long cnt = (long long)q.m_tiles * q.n_tiles * q.splits;
+    if (cnt + items > 0x3fffffff) return TEMPLORA_ERR_UNSUPPORTED;
+    items += (int)cnt;
+    bool ok = make_operand_map(&q.tmA, p.A, p.M, p.K, p.lda, p.a_mn, BM) &&
+              make_operand_map(&q.tmB, p.B, p.N, p.K, p.ldb, p.b_mn, BN);
+    if (p.Kext > 0) {
+      if (!p.Aext || !p.Bext || ((p.ldaext | p.ldbext) & 7)) return TEMPLORA_ERR_INVALID_ARG;
+      ok = ok && make_operand_map(&q.tmAe, p.Aext, p.M, p.Kext, p.ldaext, p.a_mn, BM) &&
+           make_operand_map(&q.tmBe, p.Bext, p.N, p.Kext, p.ldbext, p.b_mn, BN);
+    } else {
+      q.tmAe = q.tmA;
+      q.tmBe = q.tmB;
+    }
+    if (!ok) return TEMPLORA_ERR_CUDA;
+  }
+  g.n_items = items;
+  if (BN == 256) return launch<256>(g, di, 0, st);
+  if (BN == 64) return launch<64>(g, di, 1, st);
+  return launch<16>(g, di, 2, st);
+}
+
+}  // namespace templora

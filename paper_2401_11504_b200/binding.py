@@ -1,0 +1,193 @@
+"""Thin Python binding over the C ABI of libtemplora.so (include/templora.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch provides device memory and streams.  The functions carry the
+names of the C entry points.  There is no CPU fallback: importing this module
+without the compiled library raises.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtemplora.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+F32, BF16 = 0, 1
+
+EXPORTS = [
+    "templora_workspace_bytes", "templora_update_block_workspace_bytes", "templora_linear_fwd",
+    "templora_linear_bwd", "templora_adamw_step", "templora_decode_fwd", "templora_update_block",
+    "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
+]
+
+
+class LinearDesc(C.Structure):
+    _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32), ("r", C.c_int32), ("s", C.c_float),
+                ("dtype", C.c_int32), ("W0", C.c_void_p), ("A", C.c_void_p), ("B", C.c_void_p)]
+
+
+class ParamDesc(C.Structure):
+    _fields_ = [("n", C.c_int64), ("master", C.c_void_p), ("m", C.c_void_p), ("v", C.c_void_p),
+                ("work", C.c_void_p), ("grad", C.c_void_p)]
+
+
+class TemploraError(RuntimeError):
+    def __init__(self, code, what):
+        self.code = code
+        super().__init__(f"{what}: {status_string(code)} (status {code})")
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2401_11504_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+    LP, PP = C.POINTER(LinearDesc), C.POINTER(ParamDesc)
+    lib.templora_workspace_bytes.restype = sz
+    lib.templora_workspace_bytes.argtypes = [LP, i32]
+    lib.templora_update_block_workspace_bytes.restype = sz
+    lib.templora_update_block_workspace_bytes.argtypes = [LP, i32, i32]
+    lib.templora_linear_fwd.restype = i32
+    lib.templora_linear_fwd.argtypes = [LP, i32, vp, vp, vp, vp, sz, vp]
+    lib.templora_linear_bwd.restype = i32
+    lib.templora_linear_bwd.argtypes = [LP, i32, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.templora_adamw_step.restype = i32
+    lib.templora_adamw_step.argtypes = [PP, i32, f32, f32, f32, f32, f32, i64, i32, vp]
+    lib.templora_decode_fwd.restype = i32
+    lib.templora_decode_fwd.argtypes = [LP, i32, vp, vp, vp, sz, vp]
+    lib.templora_update_block.restype = i32
+    lib.templora_update_block.argtypes = [LP, PP, PP, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                          C.POINTER(vp), i32, f32, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_status_string.restype = C.c_char_p
+    lib.templora_status_string.argtypes = [i32]
+    lib.templora_read_device_status.restype = i32
+    lib.templora_read_device_status.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i32)]
+    lib.templora_set_kernel_path.restype = i32
+    lib.templora_set_kernel_path.argtypes = [i32]
+    return lib
+
+
+lib = _load()
+
+
+def status_string(code):
+    return lib.templora_status_string(int(code)).decode()
+
+
+def _check(code, what):
+    if code != OK:
+        raise TemploraError(code, what)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def dtype_code(t):
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported storage dtype {t.dtype}")
+
+
+def linear_desc(W0, A, B, s):
+    """templora_linear_t for contiguous device tensors W0 [d_out,d_in], A [r,d_in], B [d_out,r]."""
+    for t in (W0, A, B):
+        if not t.is_contiguous():
+            raise ValueError("W0, A and B must be contiguous")
+    d_out, d_in = W0.shape
+    r = A.shape[0]
+    if tuple(A.shape) != (r, d_in) or tuple(B.shape) != (d_out, r) or A.dtype != W0.dtype or B.dtype != W0.dtype:
+        raise ValueError("shape/dtype mismatch between W0, A and B")
+    return LinearDesc(d_in, d_out, r, float(s), dtype_code(W0), W0.data_ptr(), A.data_ptr(), B.data_ptr())
+
+
+def param_desc(master, m, v, grad, work=None):
+    return ParamDesc(master.numel(), master.data_ptr(), m.data_ptr(), v.data_ptr(),
+                     0 if work is None else work.data_ptr(), grad.data_ptr())
+
+
+def templora_workspace_bytes(lin, T):
+    return int(lib.templora_workspace_bytes(C.byref(lin), int(T)))
+
+
+def templora_update_block_workspace_bytes(lins, T):
+    arr = (LinearDesc * len(lins))(*lins)
+    return int(lib.templora_update_block_workspace_bytes(arr, len(lins), int(T)))
+
+
+def alloc_workspace(nbytes, device="cuda"):
+    """Zeroed workspace (the head holds the device status record)."""
+    if nbytes <= 0:
+        raise ValueError("workspace size query failed (invalid projection?)")
+    return torch.zeros(int(nbytes), dtype=torch.uint8, device=device)
+
+
+def templora_linear_fwd(lin, x, y, ws, U_save=None, stream=None):
+    _check(lib.templora_linear_fwd(C.byref(lin), x.shape[0], _ptr(x), _ptr(y), _ptr(U_save), _ptr(ws),
+                                   ws.numel(), _stream(stream)), "templora_linear_fwd")
+
+
+def templora_linear_bwd(lin, x, dY, dX, dA, dB, ws, U_saved=None, accumulate=False, stream=None):
+    _check(lib.templora_linear_bwd(C.byref(lin), x.shape[0], _ptr(x), _ptr(dY), _ptr(U_saved), _ptr(dX), _ptr(dA),
+                                   _ptr(dB), int(bool(accumulate)), _ptr(ws), ws.numel(), _stream(stream)),
+           "templora_linear_bwd")
+
+
+def templora_adamw_step(params, lr, beta1, beta2, eps, weight_decay, step, work_dtype=BF16, stream=None):
+    arr = (ParamDesc * len(params))(*params)
+    _check(lib.templora_adamw_step(arr, len(params), lr, beta1, beta2, eps, weight_decay, int(step),
+                                   int(work_dtype), _stream(stream)), "templora_adamw_step")
+
+
+def templora_decode_fwd(lin, x, y, ws, stream=None):
+    _check(lib.templora_decode_fwd(C.byref(lin), x.shape[0], _ptr(x), _ptr(y), _ptr(ws), ws.numel(),
+                                   _stream(stream)), "templora_decode_fwd")
+
+
+class UpdateBlockArgs:
+    """Marshalled argument arrays of templora_update_block, built once and reusable."""
+
+    def __init__(self, lins, A_states, B_states, xs, dYs, ys, dXs=None):
+        n = len(lins)
+        self.n = n
+        self.T = xs[0].shape[0]
+        self.lins = (LinearDesc * n)(*lins)
+        self.A = (ParamDesc * n)(*A_states)
+        self.B = (ParamDesc * n)(*B_states)
+        vp = C.c_void_p
+        self.x = (vp * n)(*[t.data_ptr() for t in xs])
+        self.dY = (vp * n)(*[t.data_ptr() for t in dYs])
+        self.y = (vp * n)(*[t.data_ptr() for t in ys])
+        self.dX = None if dXs is None else (vp * n)(*[0 if t is None else t.data_ptr() for t in dXs])
+        self._keep = (lins, A_states, B_states, xs, dYs, ys, dXs)
+
+
+def templora_update_block(args, epochs, lr, beta1, beta2, eps, weight_decay, step, ws, stream=None):
+    """Runs the chunk update; returns the new optimizer step count."""
+    st = C.c_int64(int(step))
+    _check(lib.templora_update_block(args.lins, args.A, args.B, args.n, args.T, args.x, args.dY, args.y, args.dX,
+                                     int(epochs), lr, beta1, beta2, eps, weight_decay, C.byref(st), _ptr(ws),
+                                     ws.numel(), _stream(stream)), "templora_update_block")
+    return st.value
+
+
+def templora_read_device_status(ws, stream=None):
+    code, where = C.c_int32(0), C.c_int32(0)
+    _check(lib.templora_read_device_status(_ptr(ws), _stream(stream), C.byref(code), C.byref(where)),
+           "templora_read_device_status")
+    return code.value, where.value
+
+
+def templora_set_kernel_path(mode):
+    return int(lib.templora_set_kernel_path(int(mode)))

@@ -1,0 +1,89 @@
+"""Helpers shared by the GPU parity tests: run the CUDA path through the C ABI on seeded
+inputs, run the fp64 oracle on the same tensors, compare per output tensor.
+
+Tolerances (per output tensor, normwise):  max|gpu - ref| <= tol * max|ref| with
+tol = 1e-2 for bf16 storage with fp32 accumulation and 1e-5 for the fp32 path.
+"""
+import numpy as np
+import torch
+
+from oracle import templora_oracle as orc
+from paper_2401_11504_b200 import inputs
+
+TOL = {"f32": 1e-5, "bf16": 1e-2}
+
+
+def tdtype(dtype):
+    return {"f32": torch.float32, "bf16": torch.bfloat16}[dtype]
+
+
+def assert_close(name, got, ref, tol):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, f"{name}: shape {got.shape} vs {ref.shape}"
+    assert np.isfinite(got).all(), f"{name}: non-finite values"
+    scale = np.abs(ref).max()
+    err = np.abs(got - ref).max()
+    assert err <= tol * scale + 1e-30, f"{name}: max|err| {err:.3e} > {tol:g} * max|ref| {scale:.3e}"
+    return err / max(scale, 1e-300)
+
+
+def f64(t):
+    return inputs.to_f64(t)
+
+
+def run_fwd_bwd(b, host, s, T, with_dX=True, save_U=True, accumulate=False):
+    """host: dict of CPU tensors (x, W0, A, B, dY).  Returns GPU outputs as float64 numpy."""
+    dev = {k: v.cuda() for k, v in host.items()}
+    d_out, d_in = host["W0"].shape
+    r = host["A"].shape[0]
+    lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], s)
+    ws = b.alloc_workspace(b.templora_workspace_bytes(lin, T))
+    dt = host["x"].dtype
+    y = torch.full((T, d_out), float("nan"), dtype=dt, device="cuda")
+    dX = torch.full((T, d_in), float("nan"), dtype=dt, device="cuda") if with_dX else None
+    U = torch.full((T, r), float("nan"), dtype=torch.float32, device="cuda") if save_U else None
+    init = 1.0 if accumulate else float("nan")
+    dA = torch.full((r, d_in), init, dtype=torch.float32, device="cuda")
+    dB = torch.full((d_out, r), init, dtype=torch.float32, device="cuda")
+    b.templora_linear_fwd(lin, dev["x"], y, ws, U_save=U)
+    b.templora_linear_bwd(lin, dev["x"], dev["dY"], dX, dA, dB, ws, U_saved=U, accumulate=accumulate)
+    code, where = b.templora_read_device_status(ws)
+    assert code == 0, f"device status {code} at {where}"
+    out = dict(y=f64(y), dA=f64(dA), dB=f64(dB))
+    if with_dX:
+        out["dX"] = f64(dX)
+    if save_U:
+        out["U"] = f64(U)
+    return out
+
+
+def oracle_fwd_bwd(host, s):
+    x, W0, A, B, dY = (f64(host[k]) for k in ("x", "W0", "A", "B", "dY"))
+    y, U = orc.linear_fwd(x, W0, A, B, s)
+    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, s)
+    return dict(y=y, U=U, dX=dX, dA=dA, dB=dB)
+
+
+def check_fwd_bwd(b, seed, tag, T, d_in, d_out, r, s, dtype, **kw):
+    host = inputs.make_linear(seed, tag, T, d_in, d_out, r, dtype=dtype, zero_B=kw.pop("zero_B", False))
+    got = run_fwd_bwd(b, host, s, T, **kw)
+    ref = oracle_fwd_bwd(host, s)
+    if kw.get("accumulate"):
+        ref["dA"] = ref["dA"] + 1.0
+        ref["dB"] = ref["dB"] + 1.0
+    errs = {}
+    for k in got:
+        errs[k] = assert_close(f"{tag}:{k}", got[k], ref[k], TOL[dtype])
+    return got, ref, errs
+
+
+def make_state(host, dtype):
+    """Device-side module state for update_block / adamw: masters, moments, grads, working copies."""
+    st = {}
+    for name in ("A", "B"):
+        master = host[name].to(torch.float32).cuda().contiguous()
+        st[name] = dict(master=master, m=torch.zeros_like(master), v=torch.zeros_like(master),
+                        grad=torch.zeros_like(master),
+                        work=master.to(torch.bfloat16).contiguous() if dtype == "bf16" else None)
+    return st

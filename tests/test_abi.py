@@ -1,0 +1,102 @@
+"""CPU-only checks of the C-ABI library: it builds, loads, exports every symbol the public
+header declares, and its host-side argument checks answer without touching a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from conftest import ROOT
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2401_11504_b200 import build
+    build.build_library()
+    from paper_2401_11504_b200 import binding
+    return binding
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "templora.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(templora_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(b):
+    names = declared_functions()
+    assert len(names) >= 10
+    raw = C.CDLL(b.LIB_PATH)
+    for n in names:
+        assert hasattr(raw, n), f"{n} declared in templora.h but not exported"
+    assert sorted(b.EXPORTS) == [n for n in names if n in b.EXPORTS]
+    for n in names:
+        assert n in b.EXPORTS, f"{n} has no Python binding"
+
+
+def test_status_strings(b):
+    seen = {b.status_string(c) for c in range(6)}
+    assert len(seen) == 6 and "ok" in seen
+    assert b.status_string(99) == "unknown status"
+
+
+def _lin(b, d_in=4096, d_out=4096, r=64, dtype=None, ptr=0x1000):
+    return b.LinearDesc(d_in, d_out, r, 2.0, b.BF16 if dtype is None else dtype, ptr, ptr, ptr)
+
+
+def test_workspace_sizes_are_sane(b):
+    lin = _lin(b)
+    n1 = b.templora_workspace_bytes(lin, 1024)
+    n2 = b.templora_workspace_bytes(lin, 2048)
+    assert 1024 < n1 < n2 < (1 << 30)
+    assert b.templora_workspace_bytes(lin, 0) == 0
+    assert b.templora_workspace_bytes(_lin(b, r=512), 128) == 0          # rank beyond 256
+    assert b.templora_workspace_bytes(_lin(b, dtype=7), 128) == 0
+    from paper_2401_11504_b200 import inputs
+    lins = [_lin(b, di, do) for _, di, do in inputs.LLAMA2_7B_BLOCK]
+    nb = b.templora_update_block_workspace_bytes(lins, 1024)
+    assert n1 <= nb < (1 << 31)
+    # a block of 32 x 7 projections needs no more than the largest group of 8
+    assert b.templora_update_block_workspace_bytes(lins * 32, 1024) <= 2 * nb
+
+
+def test_argument_errors_are_synchronous(b):
+    lib = b.lib
+    lin = _lin(b)
+    vp = C.c_void_p
+    # NULL tensors, zero rows, bad token counts, missing workspace: all rejected before any launch
+    assert lib.templora_linear_fwd(C.byref(lin), 16, None, None, None, None, 0, None) == b.ERR_INVALID_ARG
+    assert lib.templora_linear_fwd(C.byref(lin), 0, vp(0x1000), vp(0x1000), None, vp(0x1000), 1 << 20, None) == b.ERR_INVALID_ARG
+    assert lib.templora_linear_fwd(C.byref(lin), 16, vp(0x1008), vp(0x1000), None, vp(0x1000), 1 << 20, None) == b.ERR_INVALID_ARG
+    assert lib.templora_linear_fwd(C.byref(lin), 16, vp(0x1000), vp(0x1000), None, None, 0, None) == b.ERR_WORKSPACE
+    assert lib.templora_linear_fwd(C.byref(lin), 16, vp(0x1000), vp(0x1000), None, vp(0x1010), 1 << 20, None) == b.ERR_WORKSPACE
+    assert lib.templora_decode_fwd(C.byref(lin), 17, vp(0x1000), vp(0x1000), vp(0x1000), 1 << 20, None) == b.ERR_INVALID_ARG
+    assert lib.templora_decode_fwd(C.byref(lin), 0, vp(0x1000), vp(0x1000), vp(0x1000), 1 << 20, None) == b.ERR_INVALID_ARG
+    bad = _lin(b, r=257)
+    assert lib.templora_linear_fwd(C.byref(bad), 16, vp(0x1000), vp(0x1000), None, vp(0x1000), 1 << 20, None) == b.ERR_UNSUPPORTED
+    assert lib.templora_linear_bwd(C.byref(lin), 16, vp(0x1000), vp(0x1000), None, None, None, None, 0,
+                                   vp(0x1000), 1 << 20, None) == b.ERR_INVALID_ARG
+    p = b.ParamDesc(16, 0x1000, 0x1000, 0x1000, 0, 0x1000)
+    arr = (b.ParamDesc * 1)(p)
+    assert lib.templora_adamw_step(arr, 1, 1e-3, 0.9, 0.999, 1e-8, 0.0, 0, b.BF16, None) == b.ERR_INVALID_ARG   # step < 1
+    assert lib.templora_adamw_step(arr, 1, 1e-3, 1.5, 0.999, 1e-8, 0.0, 1, b.BF16, None) == b.ERR_INVALID_ARG   # beta1
+    assert lib.templora_adamw_step(None, 1, 1e-3, 0.9, 0.999, 1e-8, 0.0, 1, b.BF16, None) == b.ERR_INVALID_ARG
+
+
+def test_update_block_rejects_unaliased_parameters(b):
+    lib = b.lib
+    lin = _lin(b, ptr=0x2000)
+    lins = (b.LinearDesc * 1)(lin)
+    A = (b.ParamDesc * 1)(b.ParamDesc(64 * 4096, 0x1000, 0x1000, 0x1000, 0x3000, 0x1000))   # work != lin.A
+    Bp = (b.ParamDesc * 1)(b.ParamDesc(64 * 4096, 0x1000, 0x1000, 0x1000, 0x2000, 0x1000))
+    vp = C.c_void_p
+    arr = (vp * 1)(0x1000)
+    step = C.c_int64(0)
+    rc = lib.templora_update_block(lins, A, Bp, 1, 16, arr, arr, arr, None, 1, 1e-3, 0.9, 0.999, 1e-8, 0.0,
+                                   C.byref(step), vp(0x1000), 1 << 20, None)
+    assert rc == b.ERR_INVALID_ARG and step.value == 0
+
+
+def test_kernel_path_switch_round_trips(b):
+    prev = b.templora_set_kernel_path(1)
+    assert b.templora_set_kernel_path(prev) == 1

@@ -1,0 +1,281 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs, element by element.  Shapes span several tiles (128-row, 64/256-column tiles,
+64-wide k-blocks) and ragged tails; the full-size workloads are in test_parity_full_gpu.py."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import templora_oracle as orc
+from paper_2401_11504_b200 import inputs
+from parity_utils import TOL, assert_close, check_fwd_bwd, f64, make_state, oracle_fwd_bwd, run_fwd_bwd
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2401_11504_b200 import build
+    build.build_library()
+    from paper_2401_11504_b200 import binding
+    assert torch.cuda.get_device_capability(0)[0] == 10, "these kernels are built for sm_100a only"
+    binding.templora_set_kernel_path(0)
+    return binding
+
+
+@pytest.fixture
+def generic_path(b):
+    b.templora_set_kernel_path(1)
+    yield b
+    b.templora_set_kernel_path(0)
+
+
+# ------------------------------------------------------------------ fp32 path (configuration 0)
+def test_config0_fp32_fwd_bwd(b):
+    c = inputs.CONFIGS[0]
+    _, d_in, d_out = c["projections"][0]
+    check_fwd_bwd(b, 0, "cfg0", c["T"], d_in, d_out, c["r"], c["s"], "f32")
+
+
+@pytest.mark.parametrize("T,d_in,d_out,r", [(1, 8, 8, 1), (37, 100, 67, 5), (130, 70, 129, 8), (64, 64, 64, 16)])
+def test_fp32_ragged_shapes(b, T, d_in, d_out, r):
+    check_fwd_bwd(b, 1, f"f32-{T}-{d_in}-{d_out}-{r}", T, d_in, d_out, r, 2.0, "f32")
+
+
+def test_fp32_options(b):
+    # no dX, U recomputed in the backward, gradients accumulated onto existing contents
+    check_fwd_bwd(b, 2, "f32-opts", 50, 96, 80, 8, 1.0, "f32", with_dX=False, save_U=False, accumulate=True)
+
+
+# ------------------------------------------------------------------ bf16, tensor-core path
+TC_SHAPES = [
+    (128, 512, 512, 64),     # exactly one row tile
+    (300, 328, 520, 24),     # ragged rows, d not a multiple of 64, rank below one k-block
+    (1, 64, 72, 8),          # a single token
+    (257, 1024, 264, 128),   # two rank k-blocks, ragged columns
+    (640, 4096, 1024, 64),   # split-K in the skinny products
+    (200, 136, 2048, 256),   # maximum rank
+]
+
+
+@pytest.mark.parametrize("T,d_in,d_out,r", TC_SHAPES)
+def test_bf16_tensor_core_shapes(b, T, d_in, d_out, r):
+    check_fwd_bwd(b, 3, f"tc-{T}-{d_in}-{d_out}-{r}", T, d_in, d_out, r, 2.0, "bf16")
+
+
+def test_bf16_tensor_core_options(b):
+    check_fwd_bwd(b, 4, "tc-opts", 384, 512, 768, 64, 1.0, "bf16", with_dX=False, save_U=False, accumulate=True)
+
+
+def test_bf16_results_are_run_to_run_identical(b):
+    host = inputs.make_linear(5, "det", 300, 512, 640, 64, dtype="bf16")
+    a = run_fwd_bwd(b, host, 2.0, 300)
+    c = run_fwd_bwd(b, host, 2.0, 300)
+    for k in a:
+        assert np.array_equal(a[k], c[k]), f"{k} differs between two runs"
+
+
+def test_zero_B_gives_base_linear_and_zero_dA(b):
+    got, ref, _ = check_fwd_bwd(b, 6, "zeroB", 200, 256, 320, 64, 2.0, "bf16", zero_B=True)
+    assert not got["dA"].any()
+
+
+# ------------------------------------------------------------------ bf16, generic path
+@pytest.mark.parametrize("T,d_in,d_out,r", [(65, 100, 36, 5), (128, 512, 512, 64), (33, 200, 136, 8)])
+def test_bf16_generic_path(generic_path, T, d_in, d_out, r):
+    check_fwd_bwd(generic_path, 7, f"gen-{T}-{d_in}-{d_out}-{r}", T, d_in, d_out, r, 2.0, "bf16")
+
+
+def test_bf16_unaligned_shape_takes_generic_path_automatically(b):
+    check_fwd_bwd(b, 8, "auto-generic", 40, 100, 60, 4, 2.0, "bf16")
+
+
+# ------------------------------------------------------------------ decode
+@pytest.mark.parametrize("n", [1, 4, 16, 7])
+@pytest.mark.parametrize("d_in,d_out,r", [(512, 640, 64), (4096, 1024, 64), (1000, 264, 16)])
+def test_decode_matches_oracle(b, n, d_in, d_out, r):
+    host = inputs.make_linear(9, f"dec-{n}-{d_in}-{d_out}", n, d_in, d_out, r, dtype="bf16")
+    dev = {k: v.cuda() for k, v in host.items()}
+    lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], 2.0)
+    ws = b.alloc_workspace(b.templora_workspace_bytes(lin, 16))
+    y = torch.full((n, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+    b.templora_decode_fwd(lin, dev["x"], y, ws)
+    assert b.templora_read_device_status(ws)[0] == 0
+    ref = orc.decode_fwd(f64(host["x"]), f64(host["W0"]), f64(host["A"]), f64(host["B"]), 2.0)
+    assert_close("decode y", f64(y), ref, TOL["bf16"])
+
+
+def test_decode_fp32_and_generic(generic_path):
+    b = generic_path
+    for dtype in ("f32", "bf16"):
+        host = inputs.make_linear(10, "dec-gen-" + dtype, 4, 96, 72, 8, dtype=dtype)
+        dev = {k: v.cuda() for k, v in host.items()}
+        lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], 2.0)
+        ws = b.alloc_workspace(b.templora_workspace_bytes(lin, 16))
+        y = torch.empty((4, 72), dtype=host["x"].dtype, device="cuda")
+        b.templora_decode_fwd(lin, dev["x"], y, ws)
+        ref = orc.decode_fwd(f64(host["x"]), f64(host["W0"]), f64(host["A"]), f64(host["B"]), 2.0)
+        assert_close("decode y", f64(y), ref, TOL[dtype])
+
+
+# ------------------------------------------------------------------ AdamW
+def _adamw_case(b, n, dtype, steps, hp, seed):
+    g = torch.Generator().manual_seed(seed)
+    p0 = (torch.randn(n, generator=g) * 0.02).float()
+    grads = [torch.randn(n, generator=g).float() * (0.5 + k) for k in range(steps)]
+    p, m, v = p0.cuda(), torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    work = torch.zeros(n, dtype=torch.bfloat16, device="cuda") if dtype == "bf16" else None
+    rp, rm, rv = f64(p0), np.zeros(n), np.zeros(n)
+    for t in range(1, steps + 1):
+        gd = grads[t - 1].cuda()
+        before = f64(p)
+        b.templora_adamw_step([b.param_desc(p, m, v, gd, work)], step=t,
+                              work_dtype=b.BF16 if dtype == "bf16" else b.F32, **hp)
+        torch.cuda.synchronize()
+        rp_new, rm, rv = orc.adamw_step(rp, f64(grads[t - 1]), rm, rv, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                        hp["weight_decay"], t)
+        assert_close("p", f64(p), rp_new, 1e-5)
+        assert_close("m", f64(m), rm, 1e-5)
+        assert_close("v", f64(v), rv, 1e-5)
+        # the step itself: |dp| ~ lr is far below |p|, so compare the deltas; fp32 storage of p
+        # adds half an ulp of |p| to each side
+        d_gpu, d_ref = f64(p) - before, rp_new - rp
+        bound = 1e-5 * np.abs(d_ref).max() + 2.0 ** -23 * np.abs(rp).max()
+        assert np.abs(d_gpu - d_ref).max() <= bound
+        assert np.abs(d_ref).max() > 0
+        if work is not None:
+            assert np.array_equal(f64(work), orc.round_bf16(f64(p).astype(np.float32)))
+        # the oracle continues from the fp32 state the device holds (storage rounding is not error)
+        rp, rm, rv = f64(p), f64(m), f64(v)
+
+
+@pytest.mark.parametrize("n", [1, 7, 4096, 64 * 4096 + 3])
+def test_adamw_matches_oracle(b, n):
+    _adamw_case(b, n, "bf16", 3, dict(inputs.ADAMW), 11)
+    _adamw_case(b, n, "f32", 2, dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1), 12)
+
+
+def test_adamw_many_tensors_one_call(b):
+    hp = dict(inputs.ADAMW)
+    sizes = [5, 64 * 512, 3, 512 * 64, 1000] * 30      # 150 tensors: several launches of 64
+    g = torch.Generator().manual_seed(13)
+    ps = [(torch.randn(n, generator=g) * 0.02).float().cuda() for n in sizes]
+    gs = [torch.randn(n, generator=g).float().cuda() for n in sizes]
+    ms = [torch.zeros(n, device="cuda") for n in sizes]
+    vs = [torch.zeros(n, device="cuda") for n in sizes]
+    ws_ = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for n in sizes]
+    p0 = [f64(p) for p in ps]
+    b.templora_adamw_step([b.param_desc(p, m, v, gd, w) for p, m, v, gd, w in zip(ps, ms, vs, gs, ws_)], step=1, **hp)
+    torch.cuda.synchronize()
+    for i in (0, 1, 63, 64, 65, 149):
+        rp, rm, rv = orc.adamw_step(p0[i], f64(gs[i]), 0 * p0[i], 0 * p0[i], hp["lr"], hp["beta1"], hp["beta2"],
+                                    hp["eps"], hp["weight_decay"], 1)
+        assert_close("p", f64(ps[i]), rp, 1e-5)
+        assert_close("v", f64(vs[i]), rv, 1e-5)
+        assert np.array_equal(f64(ws_[i]), orc.round_bf16(f64(ps[i]).astype(np.float32)))
+
+
+# ------------------------------------------------------------------ update_block
+def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True):
+    hosts = [inputs.make_linear(seed, f"ub{i}", T, di, do, r, dtype=dtype) for i, (di, do) in enumerate(shapes)]
+    devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
+    states = [make_state(h, dtype) for h in hosts]
+    lins, As, Bs, ys, dXs = [], [], [], [], []
+    for h, d, st in zip(hosts, devs, states):
+        a = st["A"]["work"] if dtype == "bf16" else st["A"]["master"]
+        bb = st["B"]["work"] if dtype == "bf16" else st["B"]["master"]
+        lins.append(b.linear_desc(d["W0"], a, bb, s))
+        As.append(b.param_desc(st["A"]["master"], st["A"]["m"], st["A"]["v"], st["A"]["grad"], st["A"]["work"]))
+        Bs.append(b.param_desc(st["B"]["master"], st["B"]["m"], st["B"]["v"], st["B"]["grad"], st["B"]["work"]))
+        ys.append(torch.full_like(d["dY"], float("nan")))
+        dXs.append(torch.full_like(d["x"], float("nan")) if with_dX else None)
+    ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(lins, T))
+    args = b.UpdateBlockArgs(lins, As, Bs, [d["x"] for d in devs], [d["dY"] for d in devs], ys,
+                             dXs if with_dX else None)
+    step = b.templora_update_block(args, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
+                                   0, ws)
+    assert b.templora_read_device_status(ws)[0] == 0
+    assert step == epochs
+    projs = [dict(x=f64(h["x"]), dY=f64(h["dY"]), W0=f64(h["W0"]), s=s, A_master=f64(h["A"]), B_master=f64(h["B"]))
+             for h in hosts]
+    ref, rstep = orc.update_block(projs, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
+                                  bf16_work=(dtype == "bf16"))
+    assert rstep == step
+    tol = TOL[dtype]
+    for i, (q, st) in enumerate(zip(ref, states)):
+        assert_close(f"y{i}", f64(ys[i]), q["y"], tol)
+        if with_dX:
+            assert_close(f"dX{i}", f64(dXs[i]), q["dX"], tol)
+        assert_close(f"dA{i}", f64(st["A"]["grad"]), q["dA"], tol)
+        assert_close(f"dB{i}", f64(st["B"]["grad"]), q["dB"], tol)
+        for nm in ("A", "B"):
+            assert_close(f"{nm}{i} master", f64(st[nm]["master"]), q[nm + "_master"], tol)
+            # The update itself (|delta| ~ epochs * lr << |p|).  Adam's step is sign-like
+            # (lr * g / (|g| + eps) at step 1), so it is ill-conditioned where |g| is below the
+            # gradient's own tolerance: there the two sides may legitimately differ by up to
+            # 2 lr.  Require agreement everywhere except on a small fraction of such elements.
+            p0 = f64(hosts[i][nm])
+            d_gpu, d_ref = f64(st[nm]["master"]) - p0, q[nm + "_master"] - p0
+            assert np.abs(d_ref).max() > 0
+            bound = tol * np.abs(d_ref).max() + 2.0 ** -23 * np.abs(q[nm + "_master"]).max()
+            outliers = np.abs(d_gpu - d_ref) > bound
+            assert outliers.mean() <= (0.02 if dtype == "bf16" else 1e-3), f"{nm}{i}: {outliers.mean():.4f} of steps off"
+            if epochs == 1:
+                # exact check of the optimizer arithmetic: the oracle's step fed with the
+                # gradient the device produced must reproduce the device's step tightly
+                g_dev = f64(st[nm]["grad"])
+                p1, _, _ = orc.adamw_step(p0, g_dev, 0 * p0, 0 * p0, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                          hp["weight_decay"], 1)
+                tight = 1e-5 * np.abs(p1 - p0).max() + 2.0 ** -23 * np.abs(p1).max()
+                assert np.abs(d_gpu - (p1 - p0)).max() <= tight
+            assert_close(f"m{nm}{i}", f64(st[nm]["m"]), q["m" + nm], tol)
+            assert_close(f"v{nm}{i}", f64(st[nm]["v"]), q["v" + nm], 2 * tol)   # v is quadratic in g
+            if dtype == "bf16":
+                assert np.array_equal(f64(st[nm]["work"]), orc.round_bf16(f64(st[nm]["master"]).astype(np.float32)))
+
+
+def test_update_block_fp32_config0(b):
+    c = inputs.CONFIGS[0]
+    _update_block_case(b, "f32", [(512, 512)], c["T"], c["r"], c["s"], 1, dict(inputs.ADAMW), 0)
+
+
+def test_update_block_bf16_two_epochs(b):
+    shapes = [(256, 256), (256, 256), (256, 704), (704, 256)]
+    _update_block_case(b, "bf16", shapes, 200, 64, 2.0, 2, dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8,
+                                                                 weight_decay=0.0), 21)
+
+
+def test_update_block_more_projections_than_one_group(b):
+    shapes = [(128, 192)] * 5 + [(192, 128)] * 6
+    _update_block_case(b, "bf16", shapes, 130, 16, 2.0, 1, dict(inputs.ADAMW), 22, with_dX=False)
+
+
+def test_update_block_generic_path(generic_path):
+    _update_block_case(generic_path, "bf16", [(100, 60), (60, 100)], 33, 4, 2.0, 2,
+                       dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01), 23)
+
+
+def test_update_block_zero_epochs_is_a_no_op(b):
+    host = inputs.make_linear(24, "noop", 16, 64, 64, 8, dtype="bf16")
+    d = {k: v.cuda() for k, v in host.items()}
+    st = make_state(host, "bf16")
+    lin = b.linear_desc(d["W0"], st["A"]["work"], st["B"]["work"], 2.0)
+    A = b.param_desc(st["A"]["master"], st["A"]["m"], st["A"]["v"], st["A"]["grad"], st["A"]["work"])
+    Bp = b.param_desc(st["B"]["master"], st["B"]["m"], st["B"]["v"], st["B"]["grad"], st["B"]["work"])
+    y = torch.zeros_like(d["dY"])
+    ws = b.alloc_workspace(b.templora_update_block_workspace_bytes([lin], 16))
+    args = b.UpdateBlockArgs([lin], [A], [Bp], [d["x"]], [d["dY"]], [y])
+    assert b.templora_update_block(args, 0, 1e-3, 0.9, 0.999, 1e-8, 0.0, 5, ws) == 5
+    torch.cuda.synchronize()
+    assert np.array_equal(f64(st["A"]["master"]), f64(host["A"]))
+
+
+# ------------------------------------------------------------------ errors that need a device
+def test_short_workspace_is_rejected(b):
+    host = inputs.make_linear(25, "short", 256, 512, 512, 64, dtype="bf16")
+    d = {k: v.cuda() for k, v in host.items()}
+    lin = b.linear_desc(d["W0"], d["A"], d["B"], 2.0)
+    ws = b.alloc_workspace(2048)
+    y = torch.empty((256, 512), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(b.TemploraError) as e:
+        b.templora_linear_fwd(lin, d["x"], y, ws)
+    assert e.value.code == b.ERR_WORKSPACE

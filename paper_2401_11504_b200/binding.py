@@ -109,12 +109,16 @@ def linear_desc(W0, A, B, s):
     r = A.shape[0]
     if tuple(A.shape) != (r, d_in) or tuple(B.shape) != (d_out, r) or A.dtype != W0.dtype or B.dtype != W0.dtype:
         raise ValueError("shape/dtype mismatch between W0, A and B")
-    return LinearDesc(d_in, d_out, r, float(s), dtype_code(W0), W0.data_ptr(), A.data_ptr(), B.data_ptr())
+    desc = LinearDesc(d_in, d_out, r, float(s), dtype_code(W0), W0.data_ptr(), A.data_ptr(), B.data_ptr())
+    desc._keep = (W0, A, B)  # the descriptor holds raw pointers: keep the tensors alive with it
+    return desc
 
 
 def param_desc(master, m, v, grad, work=None):
-    return ParamDesc(master.numel(), master.data_ptr(), m.data_ptr(), v.data_ptr(),
+    desc = ParamDesc(master.numel(), master.data_ptr(), m.data_ptr(), v.data_ptr(),
                      0 if work is None else work.data_ptr(), grad.data_ptr())
+    desc._keep = (master, m, v, grad, work)
+    return desc
 
 
 def templora_workspace_bytes(lin, T):

@@ -13,6 +13,12 @@ from paper_2401_11504_b200 import inputs
 TOL = {"f32": 1e-5, "bf16": 1e-2}
 
 
+def hp32(hp):
+    """Optimizer hyper-parameters as the C ABI receives them: rounded to fp32 (1 - beta2 changes by
+    1.3e-5 relative when 0.999 is rounded to fp32; both sides must see the same value)."""
+    return {k: float(np.float32(v)) for k, v in hp.items()}
+
+
 def tdtype(dtype):
     return {"f32": torch.float32, "bf16": torch.bfloat16}[dtype]
 

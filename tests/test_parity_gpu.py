@@ -7,7 +7,7 @@ import torch
 
 from oracle import templora_oracle as orc
 from paper_2401_11504_b200 import inputs
-from parity_utils import TOL, assert_close, check_fwd_bwd, f64, make_state, oracle_fwd_bwd, run_fwd_bwd
+from parity_utils import TOL, assert_close, check_fwd_bwd, f64, hp32, make_state, oracle_fwd_bwd, run_fwd_bwd
 
 pytestmark = pytest.mark.gpu
 
@@ -119,6 +119,7 @@ def test_decode_fp32_and_generic(generic_path):
 
 # ------------------------------------------------------------------ AdamW
 def _adamw_case(b, n, dtype, steps, hp, seed):
+    hp = hp32(hp)
     g = torch.Generator().manual_seed(seed)
     p0 = (torch.randn(n, generator=g) * 0.02).float()
     grads = [torch.randn(n, generator=g).float() * (0.5 + k) for k in range(steps)]
@@ -155,7 +156,7 @@ def test_adamw_matches_oracle(b, n):
 
 
 def test_adamw_many_tensors_one_call(b):
-    hp = dict(inputs.ADAMW)
+    hp = hp32(inputs.ADAMW)
     sizes = [5, 64 * 512, 3, 512 * 64, 1000] * 30      # 150 tensors: several launches of 64
     g = torch.Generator().manual_seed(13)
     ps = [(torch.randn(n, generator=g) * 0.02).float().cuda() for n in sizes]
@@ -176,6 +177,7 @@ def test_adamw_many_tensors_one_call(b):
 
 # ------------------------------------------------------------------ update_block
 def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True):
+    hp = hp32(hp)
     hosts = [inputs.make_linear(seed, f"ub{i}", T, di, do, r, dtype=dtype) for i, (di, do) in enumerate(shapes)]
     devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
     states = [make_state(h, dtype) for h in hosts]
@@ -208,7 +210,10 @@ def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True
         assert_close(f"dA{i}", f64(st["A"]["grad"]), q["dA"], tol)
         assert_close(f"dB{i}", f64(st["B"]["grad"]), q["dB"], tol)
         for nm in ("A", "B"):
-            assert_close(f"{nm}{i} master", f64(st[nm]["master"]), q[nm + "_master"], tol)
+            # master parameters: within tolerance, plus the worst case of the sign-like Adam step on
+            # elements whose gradient is below its own tolerance (2 lr per epoch, see below)
+            err = np.abs(f64(st[nm]["master"]) - q[nm + "_master"]).max()
+            assert err <= tol * np.abs(q[nm + "_master"]).max() + 2.0 * epochs * hp["lr"]
             # The update itself (|delta| ~ epochs * lr << |p|).  Adam's step is sign-like
             # (lr * g / (|g| + eps) at step 1), so it is ill-conditioned where |g| is below the
             # gradient's own tolerance: there the two sides may legitimately differ by up to

@@ -163,6 +163,24 @@ templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *c
  */
 int32_t templora_set_kernel_path(int32_t mode);
 
+/*
+ * Launch accounting, a profiling aid (the paper has no counterpart).  The library counts
+ * the launches of each kernel class; with timing enabled it also records a pair of CUDA
+ * events on the launching stream around every launch.  Kernel classes: 0 tensor-core GEMM
+ * with 256-wide tiles (y, dX), 1 tensor-core GEMM with 64-wide tiles (U, V, dA, dB),
+ * 2 tensor-core GEMM with 16-wide tiles (decode), 3 partial reduction, 4 AdamW,
+ * 5 generic GEMM, 6 decode finish.  Process-wide.
+ */
+void templora_timing_enable(int32_t on);
+
+/*
+ * Waits for the recorded events of class `kind` and returns their summed device time
+ * (*total_ms), how many launches were timed and how many were counted since the last
+ * reset.  reset != 0 clears the class afterwards.  Output pointers may be NULL.
+ */
+templora_status_t templora_timing_read(int32_t kind, double *total_ms, int64_t *timed_launches,
+                                       int64_t *all_launches, int32_t reset);
+
 #ifdef __cplusplus
 }
 #endif

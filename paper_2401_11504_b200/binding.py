@@ -20,7 +20,10 @@ EXPORTS = [
     "templora_workspace_bytes", "templora_update_block_workspace_bytes", "templora_linear_fwd",
     "templora_linear_bwd", "templora_adamw_step", "templora_decode_fwd", "templora_update_block",
     "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
+    "templora_timing_enable", "templora_timing_read",
 ]
+KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH = range(7)
+N_KINDS = 7
 
 
 class LinearDesc(C.Structure):
@@ -67,6 +70,10 @@ def _load():
     lib.templora_read_device_status.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i32)]
     lib.templora_set_kernel_path.restype = i32
     lib.templora_set_kernel_path.argtypes = [i32]
+    lib.templora_timing_enable.restype = None
+    lib.templora_timing_enable.argtypes = [i32]
+    lib.templora_timing_read.restype = i32
+    lib.templora_timing_read.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(i64), i32]
     return lib
 
 
@@ -195,3 +202,15 @@ def templora_read_device_status(ws, stream=None):
 
 def templora_set_kernel_path(mode):
     return int(lib.templora_set_kernel_path(int(mode)))
+
+
+def templora_timing_enable(on):
+    lib.templora_timing_enable(int(bool(on)))
+
+
+def templora_timing_read(kind, reset=False):
+    """-> (total_ms, timed_launches, all_launches) of one kernel class."""
+    ms, timed, allc = C.c_double(0.0), C.c_int64(0), C.c_int64(0)
+    _check(lib.templora_timing_read(int(kind), C.byref(ms), C.byref(timed), C.byref(allc), int(bool(reset))),
+           "templora_timing_read")
+    return ms.value, timed.value, allc.value

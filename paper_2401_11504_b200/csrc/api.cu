@@ -322,9 +322,12 @@ templora_status_t decode_impl(const templora_linear_t *l, int n, const void *x, 
     p[1].splits = spu; p[1].out = Pu; p[1].out_f32 = 1; p[1].out_s0 = 1; p[1].out_s1 = l->r;
     p[1].out_split = (long long)n * l->r;
     TL_TRY(tc_gemm_grouped(p, 2, 16, ws.status(), st));
-    decode_finish_kernel<<<cdiv(l->d_out, kFinThreads), kFinThreads, (size_t)n * l->r * sizeof(float), st>>>(
-        P, sp, Pu, spu, n, l->d_out, l->r, l->s, reinterpret_cast<const __nv_bfloat16 *>(l->B),
-        reinterpret_cast<__nv_bfloat16 *>(y));
+    {
+      LaunchScope scope(kKindDecodeFinish, st);
+      decode_finish_kernel<<<cdiv(l->d_out, kFinThreads), kFinThreads, (size_t)n * l->r * sizeof(float), st>>>(
+          P, sp, Pu, spu, n, l->d_out, l->r, l->s, reinterpret_cast<const __nv_bfloat16 *>(l->B),
+          reinterpret_cast<__nv_bfloat16 *>(y));
+    }
     TL_CUDA_CHECK(cudaGetLastError());
     return TEMPLORA_OK;
   }

@@ -35,6 +35,30 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
     if (_s != TEMPLORA_OK) return _s;                         \
   } while (0)
 
+// ---- launch accounting (timing.cu) -------------------------------------------
+enum KernelKind {
+  kKindTcMain = 0,     // tensor-core GEMM, 256-wide tiles: y and dX with the rank-r term fused
+  kKindTcSkinny = 1,   // tensor-core GEMM, 64-wide tiles: U, V, dB, dA
+  kKindTcDecode = 2,   // tensor-core GEMM, 16-wide tiles: decode-time W0 stream
+  kKindReduce = 3,     // split-K partial reduction / bf16 re-encoding
+  kKindAdamW = 4,
+  kKindSimt = 5,       // generic-shape GEMM
+  kKindDecodeFinish = 6,
+  kKindCount = 7
+};
+// Construct right before a kernel launch and destroy right after it.
+class LaunchScope {
+ public:
+  LaunchScope(int kind, cudaStream_t st);
+  ~LaunchScope();
+  LaunchScope(const LaunchScope &) = delete;
+  LaunchScope &operator=(const LaunchScope &) = delete;
+ private:
+  int kind_;
+  cudaStream_t st_;
+  cudaEvent_t a_, b_;
+};
+
 // ---- generic (SIMT) GEMM:  D = alpha1 * A1 B1 + alpha2 * A2 B2 (+ D) --------
 // Element (i,k) of an operand lives at p[i*s0 + k*s1]; dt is a templora_dtype_t.
 struct Operand {

@@ -128,7 +128,10 @@ templora_status_t reduce_partials_batch(const ReduceJob *jobs, int n_jobs, cudaS
       blocks += (int)((b.job[j].n + kRedPerBlock - 1) / kRedPerBlock);
     }
     b.block_start[b.n_jobs] = blocks;
-    reduce_partials_kernel<<<blocks, kRedThreads, 0, st>>>(b);
+    {
+      LaunchScope scope(kKindReduce, st);
+      reduce_partials_kernel<<<blocks, kRedThreads, 0, st>>>(b);
+    }
     TL_CUDA_CHECK(cudaGetLastError());
   }
   return TEMPLORA_OK;
@@ -159,7 +162,10 @@ templora_status_t adamw_launch(const templora_param_t *params, int n_params, flo
     }
     if (blocks > 0x7fffffffLL) return TEMPLORA_ERR_UNSUPPORTED;
     b.block_start[b.n_tensors] = (int)blocks;
-    adamw_kernel<<<(unsigned)blocks, kAdamThreads, 0, st>>>(b);
+    {
+      LaunchScope scope(kKindAdamW, st);
+      adamw_kernel<<<(unsigned)blocks, kAdamThreads, 0, st>>>(b);
+    }
     TL_CUDA_CHECK(cudaGetLastError());
   }
   return TEMPLORA_OK;

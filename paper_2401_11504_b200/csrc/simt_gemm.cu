@@ -90,7 +90,10 @@ templora_status_t simt_gemm(const SimtGemm &g, cudaStream_t st) {
   if (g.M <= 0 || g.N <= 0 || g.K1 <= 0) return TEMPLORA_ERR_INVALID_ARG;
   dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM);
   if (grid.y > 65535u) return TEMPLORA_ERR_UNSUPPORTED;
-  simt_gemm_kernel<<<grid, NT, 0, st>>>(g);
+  {
+    LaunchScope scope(kKindSimt, st);
+    simt_gemm_kernel<<<grid, NT, 0, st>>>(g);
+  }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;
 }

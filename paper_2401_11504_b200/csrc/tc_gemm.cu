@@ -460,7 +460,10 @@ templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream
     di->attr_set[slot] = true;
   }
   int grid = g.n_items < di->sm_count ? g.n_items : di->sm_count;
-  tc_gemm_kernel<BN><<<grid, kThreads, Cfg<BN>::kSmemBytes, st>>>(g);
+  {
+    LaunchScope scope(BN == 256 ? kKindTcMain : (BN == 64 ? kKindTcSkinny : kKindTcDecode), st);
+    tc_gemm_kernel<BN><<<grid, kThreads, Cfg<BN>::kSmemBytes, st>>>(g);
+  }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;
 }

@@ -1,0 +1,181 @@
+"""Host-side plumbing around the library: building a block of LoRA-augmented projections on a
+device, rank bookkeeping for replicated runs, and clock sampling.  No arithmetic of the method.
+
+Multi-GPU: the path does not shard (one GPU holds a whole block and its chunk); N GPUs run N
+independent replicas.  The only cross-rank steps are a barrier around the timed region and a max
+over ranks of the measured time, both through torch.distributed (nccl on GPUs, gloo on CPU).
+"""
+import os
+import threading
+import time
+
+import torch
+import torch.distributed as dist
+
+from . import inputs
+
+
+# ------------------------------------------------------------------ ranks
+class Ranks:
+    """World bookkeeping for replicated runs; a single process is world_size 1 without a group."""
+
+    def __init__(self, backend=None):
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.group = False
+        if self.world > 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29531")
+            backend = backend or ("nccl" if torch.cuda.is_available() else "gloo")
+            if backend == "nccl":
+                torch.cuda.set_device(self.local_rank)
+            dist.init_process_group(backend=backend, rank=self.rank, world_size=self.world)
+            self.group = True
+            self.backend = backend
+
+    def _dev(self):
+        return torch.device("cuda", self.local_rank) if self.group and self.backend == "nccl" else torch.device("cpu")
+
+    def barrier(self):
+        if self.group:
+            dist.barrier()
+
+    def max_over_ranks(self, value):
+        if not self.group:
+            return float(value)
+        t = torch.tensor([float(value)], dtype=torch.float64, device=self._dev())
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(self, value):
+        if not self.group:
+            return float(value)
+        t = torch.tensor([float(value)], dtype=torch.float64, device=self._dev())
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    def close(self):
+        if self.group:
+            dist.destroy_process_group()
+            self.group = False
+
+
+def aggregate_throughput(units_per_rank, seconds_this_rank, ranks):
+    """Whole-job throughput of replicated work: units of all ranks / slowest rank's time."""
+    total_units = ranks.sum_over_ranks(units_per_rank)
+    slowest = ranks.max_over_ranks(seconds_this_rank)
+    return total_units / slowest, slowest
+
+
+# ------------------------------------------------------------------ block construction
+class Block:
+    """One block of LoRA-augmented projections resident on a device, with optimizer state."""
+
+    def __init__(self, b, seed, tag, projections, T, r, s, dtype="bf16", device="cuda", with_dX=True,
+                 shared_io=None):
+        self.T, self.r, self.s, self.dtype = T, r, s, dtype
+        self.names = [p[0] for p in projections]
+        self.W0, self.state, self.lins, self.A_desc, self.B_desc = [], [], [], [], []
+        self.x, self.dY, self.y, self.dX = [], [], [], []
+        self.io = {}
+        td = torch.bfloat16 if dtype == "bf16" else torch.float32
+        for name, d_in, d_out in projections:
+            t = f"{tag}/{name}"
+            W0 = inputs.make_tensor(seed, t, "W0", (d_out, d_in), "normal", d_in ** -0.5, dtype, device)
+            st = {}
+            for nm, shape, kind, scale in (("A", (r, d_in), "uniform", d_in ** -0.5), ("B", (d_out, r), "normal", 0.02)):
+                w = inputs.make_tensor(seed, t, nm, shape, kind, scale, dtype, device)
+                master = w.float().contiguous()
+                st[nm] = dict(master=master, m=torch.zeros_like(master), v=torch.zeros_like(master),
+                              grad=torch.zeros_like(master), work=w.contiguous() if dtype == "bf16" else None)
+            a = st["A"]["work"] if dtype == "bf16" else st["A"]["master"]
+            bb = st["B"]["work"] if dtype == "bf16" else st["B"]["master"]
+            self.W0.append(W0)
+            self.state.append(st)
+            self.lins.append(b.linear_desc(W0, a, bb, s))
+            self.A_desc.append(b.param_desc(st["A"]["master"], st["A"]["m"], st["A"]["v"], st["A"]["grad"], st["A"]["work"]))
+            self.B_desc.append(b.param_desc(st["B"]["master"], st["B"]["m"], st["B"]["v"], st["B"]["grad"], st["B"]["work"]))
+            if shared_io is not None:
+                io = shared_io[name]
+            else:
+                io = dict(x=inputs.make_tensor(seed, t, "x", (T, d_in), "normal", 1.0, dtype, device),
+                          dY=inputs.make_tensor(seed, t, "dY", (T, d_out), "normal", 1.0, dtype, device))
+                io["y"] = torch.empty((T, d_out), dtype=td, device=device)
+                io["dX"] = torch.empty((T, d_in), dtype=td, device=device) if with_dX else None
+            self.io[name] = io
+            self.x.append(io["x"]); self.dY.append(io["dY"]); self.y.append(io["y"]); self.dX.append(io["dX"])
+        self.args = b.UpdateBlockArgs(self.lins, self.A_desc, self.B_desc, self.x, self.dY, self.y,
+                                      self.dX if with_dX else None)
+
+    def n_lora_params(self):
+        return sum(st["A"]["master"].numel() + st["B"]["master"].numel() for st in self.state)
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+
+    def __init__(self, cuda_index=0, period_s=0.02):
+        self.index, self.period = cuda_index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:  # NVML numbers GPUs by PCI order, CUDA by visibility: match on the PCI address
+                pr = torch.cuda.get_device_properties(cuda_index)
+                bus_id = f"{pr.pci_domain_id:08X}:{pr.pci_bus_id:02X}:{pr.pci_device_id:02X}.0"
+                self._h = pynvml.nvmlDeviceGetHandleByPciBusId(bus_id.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(cuda_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    _REASONS = (("hw_slowdown", 0x8), ("sw_power_cap", 0x4), ("hw_thermal_slowdown", 0x40),
+                ("sw_thermal_slowdown", 0x20), ("hw_power_brake", 0x80), ("sync_boost", 0x10))
+
+    def _once(self):
+        nv = self._nv
+        self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+        try:
+            mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+        except Exception:
+            mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+        for name, bit in self._REASONS:
+            if mask & bit:
+                self.reasons.add(name)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self._once()
+            except Exception:
+                break
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2.0)
+            try:
+                self._once()
+            except Exception:
+                pass
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["clock sampling unavailable"]}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}

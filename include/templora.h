@@ -164,6 +164,32 @@ templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *c
 int32_t templora_set_kernel_path(int32_t mode);
 
 /*
+ * templora_decode_fwd for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a deployment convenience).  Some hosts of this library are handed
+ * only input and output buffers and may not call cudaMalloc themselves: a serving loop whose
+ * device memory belongs entirely to another framework's pool, a latency-critical thread for
+ * which an allocation (which may synchronise the device) is off limits, a plug-in without an
+ * allocator.  This variant takes no workspace.  Its split-K scratch is a fixed array of
+ * TEMPLORA_NOALLOC_SCRATCH_BYTES inside the library image, present on every GPU that loads
+ * the library for the life of the process.  The call allocates and frees nothing.
+ *   - Same arguments and result as templora_decode_fwd, minus the workspace.
+ *   - A projection whose decode scratch would exceed the array is refused with
+ *     TEMPLORA_ERR_UNSUPPORTED and nothing is launched (all Llama-2 7B- and 70B-shaped
+ *     projections at rank 64 fit).
+ *   - The first call on each device looks up the array's device address; make that first
+ *     call with the device current and before starting any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents
+ *     (the call clears the part that must start at zero).  Two calls that may overlap on the
+ *     GPU, e.g. on different streams, race on it: serialise them, or use templora_decode_fwd
+ *     with one workspace per stream.
+ *   - The device status record of this variant lives in the array and is cleared at the start
+ *     of each call; templora_read_device_status cannot reach it.
+ */
+#define TEMPLORA_NOALLOC_SCRATCH_BYTES (8u << 20)
+templora_status_t templora_decode_fwd_noalloc(const templora_linear_t *lin, int32_t n_tokens, const void *x,
+                                              void *y, void *stream);
+
+/*
  * Launch accounting, a profiling aid (the paper has no counterpart).  The library counts
  * the launches of each kernel class; with timing enabled it also records a pair of CUDA
  * events on the launching stream around every launch.  Kernel classes: 0 tensor-core GEMM

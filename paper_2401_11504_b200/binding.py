@@ -20,8 +20,9 @@ EXPORTS = [
     "templora_workspace_bytes", "templora_update_block_workspace_bytes", "templora_linear_fwd",
     "templora_linear_bwd", "templora_adamw_step", "templora_decode_fwd", "templora_update_block",
     "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
-    "templora_timing_enable", "templora_timing_read",
+    "templora_timing_enable", "templora_timing_read", "templora_decode_fwd_noalloc",
 ]
+NOALLOC_SCRATCH_BYTES = 8 << 20
 KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH = range(7)
 N_KINDS = 7
 
@@ -70,6 +71,8 @@ def _load():
     lib.templora_read_device_status.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i32)]
     lib.templora_set_kernel_path.restype = i32
     lib.templora_set_kernel_path.argtypes = [i32]
+    lib.templora_decode_fwd_noalloc.restype = i32
+    lib.templora_decode_fwd_noalloc.argtypes = [LP, i32, vp, vp, vp]
     lib.templora_timing_enable.restype = None
     lib.templora_timing_enable.argtypes = [i32]
     lib.templora_timing_read.restype = i32
@@ -214,3 +217,11 @@ def templora_timing_read(kind, reset=False):
     _check(lib.templora_timing_read(int(kind), C.byref(ms), C.byref(timed), C.byref(allc), int(bool(reset))),
            "templora_timing_read")
     return ms.value, timed.value, allc.value
+
+
+def templora_decode_fwd_noalloc(lin, x, y, stream=None):
+    """Decode-time forward without a caller workspace: for hosts that may not allocate device
+    memory.  Scratch is a fixed array inside the library (NOALLOC_SCRATCH_BYTES per GPU), shared by
+    all calls on the device, so calls that could overlap on the GPU must be serialised."""
+    _check(lib.templora_decode_fwd_noalloc(C.byref(lin), x.shape[0], _ptr(x), _ptr(y), _stream(stream)),
+           "templora_decode_fwd_noalloc")

@@ -459,6 +459,22 @@ templora_status_t update_impl(const templora_linear_t *proj, const templora_para
 }
 
 }  // namespace
+
+// Workspace bytes that templora_decode_fwd alone needs for n tokens (0 on an invalid projection);
+// holds for either kernel path.
+size_t decode_workspace_need(const templora_linear_t *lin, int n) {
+  if (check_linear(lin) != TEMPLORA_OK || n < 1 || n > 16) return 0;
+  size_t need = kStatusBytes;
+  for (int mode = 0; mode < 2; ++mode) {
+    t_path_override = mode;
+    WsAlloc c(nullptr, 0);
+    decode_impl(lin, n, nullptr, nullptr, c, true, nullptr);
+    if (c.off > need) need = c.off;
+  }
+  t_path_override = -1;
+  return need;
+}
+
 }  // namespace templora
 
 using namespace templora;

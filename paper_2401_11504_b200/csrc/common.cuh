@@ -118,4 +118,7 @@ constexpr int kTcMaxProblems = 16;
 templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st);
 bool tc_available();
 
+// ---- workspace need of the decode-time forward alone (api.cu) -------------------
+size_t decode_workspace_need(const templora_linear_t *lin, int n);
+
 }  // namespace templora

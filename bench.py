@@ -155,12 +155,13 @@ def run_ours(args):
     hp = {k: float(v) for k, v in inputs.ADAMW.items()}
     peaks = load_peaks()
 
-    blocks = [runtime.Block(b, 0, f"r{ranks.rank}/blk{i}", projections, T, r, s, "bf16", dev) for i in range(N_ROTATE)]
+    blocks = [runtime.Block(b, 0, f"r{ranks.rank}/blk{i}", projections, T, r, s, "bf16", dev) for i in range(args.blocks)]
+    N_ROT = args.blocks
     ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(blocks[0].lins, T), dev)
-    steps_taken = [0] * N_ROTATE
+    steps_taken = [0] * N_ROT
 
     def step(i):
-        k = i % N_ROTATE
+        k = i % N_ROT
         steps_taken[k] = b.templora_update_block(blocks[k].args, 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
                                                  hp["weight_decay"], steps_taken[k], ws)
 
@@ -257,7 +258,7 @@ def run_ours(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks.world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * slowest / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "l2": f"steps rotate over {N_ROTATE} blocks with distinct weights; each block's W0 is 405 MB (> 126 MB L2)",
+                "config": {"workload": WORKLOAD, "l2": f"steps rotate over {N_ROT} blocks with distinct weights; each block's W0 is 405 MB (> 126 MB L2)",
                            "parallelism": "replicas only" if ranks.world > 1 else "single GPU",
                            "step_tflops": tf_block, "step_frac_of_measured_sustained": tf_block / ranks.world / peaks["tflops"],
                            "step_frac_of_nominal_2250": tf_block / ranks.world / 2250.0},
@@ -322,6 +323,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--blocks", type=int, default=N_ROTATE, help="distinct blocks the steps rotate over")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -93,3 +93,40 @@ def make_state(host, dtype):
                         grad=torch.zeros_like(master),
                         work=master.to(torch.bfloat16).contiguous() if dtype == "bf16" else None)
     return st
+
+
+def snapshot_block(blk):
+    """Host fp64 copies of everything the oracle needs from a runtime.Block, taken BEFORE the update."""
+    projs = []
+    for i, st in enumerate(blk.state):
+        projs.append(dict(x=f64(blk.x[i]), dY=f64(blk.dY[i]), W0=f64(blk.W0[i]), s=blk.s,
+                          A_master=f64(st["A"]["master"]), B_master=f64(st["B"]["master"]),
+                          mA=f64(st["A"]["m"]), vA=f64(st["A"]["v"]), mB=f64(st["B"]["m"]), vB=f64(st["B"]["v"])))
+    return projs
+
+
+def compare_block(blk, projs0, ref, epochs, lr, tol=1e-2, check_io=True):
+    """Device state of a block after templora_update_block against the oracle's update_block."""
+    worst = {}
+    for i, (q, st) in enumerate(zip(ref, blk.state)):
+        name = blk.names[i]
+        if check_io:
+            worst[f"{name}.y"] = assert_close(f"{name}.y", f64(blk.y[i]), q["y"], tol)
+            if blk.dX[i] is not None:
+                worst[f"{name}.dX"] = assert_close(f"{name}.dX", f64(blk.dX[i]), q["dX"], tol)
+        worst[f"{name}.dA"] = assert_close(f"{name}.dA", f64(st["A"]["grad"]), q["dA"], tol)
+        worst[f"{name}.dB"] = assert_close(f"{name}.dB", f64(st["B"]["grad"]), q["dB"], tol)
+        for nm in ("A", "B"):
+            p0 = projs0[i][nm + "_master"]
+            got = f64(st[nm]["master"])
+            err = np.abs(got - q[nm + "_master"]).max()
+            assert err <= tol * np.abs(q[nm + "_master"]).max() + 2.0 * epochs * lr, f"{name}.{nm} master"
+            d_gpu, d_ref = got - p0, q[nm + "_master"] - p0
+            assert np.abs(d_ref).max() > 0
+            bound = tol * np.abs(d_ref).max() + 2.0 ** -23 * np.abs(q[nm + "_master"]).max()
+            frac = (np.abs(d_gpu - d_ref) > bound).mean()
+            assert frac <= 0.02, f"{name}.{nm}: {frac:.4f} of the optimizer steps are off"
+            assert_close(f"{name}.m{nm}", f64(st[nm]["m"]), q["m" + nm], tol)
+            assert_close(f"{name}.v{nm}", f64(st[nm]["v"]), q["v" + nm], 2 * tol)
+            assert np.array_equal(f64(st[nm]["work"]), orc.round_bf16(got.astype(np.float32))), f"{name}.{nm} work copy"
+    return worst

@@ -14,7 +14,9 @@ namespace templora {
 struct DeviceStatus {
   int32_t code;
   int32_t where;
-  int32_t pad[62];
+  int32_t sched_next;   // tensor-core kernel: next work item to hand out (zero between launches)
+  int32_t sched_done;   // tensor-core kernel: CTAs that have finished (zero between launches)
+  int32_t pad[60];
 };
 static_assert(sizeof(DeviceStatus) == 256, "status record is 256 bytes");
 

@@ -13,6 +13,11 @@
 // tile overlap the mainloop of the next.  Every mbarrier wait is bounded: when a wait runs out the
 // CTA records TEMPLORA_ERR_TIMEOUT in the device status record, drains what it has in flight,
 // frees its TMEM and returns.
+//
+// Work items (problem, m-tile, n-tile, k-split) are drawn from a counter in the status record at the
+// head of the workspace: CTA b starts with item b and then takes "next" atomically, so the tail of
+// a launch is balanced whatever the mix of long and short items.  The counter must be zero at
+// launch (the workspace head is zeroed once by the caller); the last CTA to finish resets it.
 #include "common.cuh"
 
 #include <cuda.h>
@@ -22,6 +27,7 @@ namespace {
 
 constexpr int BM = 128, BK = 64;
 constexpr int kThreads = 192;
+constexpr int kSched = 4;  // depth of the work-item ring between the producer and its consumers
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 constexpr int kStageA = BM * BK * 2;  // 16 KB
@@ -236,6 +242,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
   const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
   volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + kStages * kStage + 512);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 516);
+  // work items are handed out dynamically: the producer draws the next item from a global counter
+  // and passes it to the MMA thread and the epilogue warps through this small ring
+  volatile int *sched_ring = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 528);
+  auto sfull_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 5 + s); };
+  auto sempty_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 5 + kSched + s); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -249,6 +260,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
       mbar_init(tempty_bar(a), 4);
     }
     mbar_init(drain_bar, 1);
+    for (int s = 0; s < kSched; ++s) {
+      mbar_init(sfull_bar(s), 1);
+      mbar_init(sempty_bar(s), 5);  // the MMA thread + one lane of each epilogue warp
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -271,7 +286,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
       uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
-      for (int item = blockIdx.x; ok && item < g.n_items; item += gridDim.x) {
+      int item = blockIdx.x, sslot = 0;
+      uint32_t sphase = 0;
+      while (ok) {
+        if (!mbar_wait(sempty_bar(sslot), sphase ^ 1u, abort_flag, g.status, 110)) { ok = false; break; }
+        sched_ring[sslot] = item;
+        mbar_arrive(sfull_bar(sslot));
+        if (++sslot == kSched) { sslot = 0; sphase ^= 1u; }
+        if (item >= g.n_items) break;  // the end marker has been passed on
+        const int next_item = (int)gridDim.x + atomicAdd(&g.status->sched_next, 1);  // drawn early, used late
         const Item it = decode_item(g, item);
         const DevProb &q = g.p[it.p];
         const int n0 = it.nt * BN;
@@ -301,6 +324,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
+        item = next_item;
       }
       if (!ok) {
         // wait (bounded) for the copies this thread still has in flight before the CTA may exit
@@ -319,9 +343,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      int local = 0;
       bool ok = true;
-      for (int item = blockIdx.x; ok && item < g.n_items; item += gridDim.x, ++local) {
+      int sslot = 0;
+      uint32_t sphase = 0;
+      for (int local = 0; ok; ++local) {
+        if (!mbar_wait(sfull_bar(sslot), sphase, abort_flag, g.status, 210)) { ok = false; break; }
+        const int item = sched_ring[sslot];
+        mbar_arrive(sempty_bar(sslot));
+        if (++sslot == kSched) { sslot = 0; sphase ^= 1u; }
+        if (item >= g.n_items) break;
         const Item it = decode_item(g, item);
         const DevProb &q = g.p[it.p];
         const int nkb = (it.kb1 - it.kb0) + it.next;
@@ -356,9 +386,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
   } else {
     // ===================== epilogue (warps 2..5) =====================
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
-    int local = 0;
     bool ok = true;
-    for (int item = blockIdx.x; ok && item < g.n_items; item += gridDim.x, ++local) {
+    int sslot = 0;
+    uint32_t sphase = 0;
+    for (int local = 0; ok; ++local) {
+      if (!mbar_wait(sfull_bar(sslot), sphase, abort_flag, g.status, 310)) { ok = false; break; }
+      const int item = sched_ring[sslot];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sempty_bar(sslot));
+      if (++sslot == kSched) { sslot = 0; sphase ^= 1u; }
+      if (item >= g.n_items) break;
       const Item it = decode_item(g, item);
       const DevProb &q = g.p[it.p];
       const int n0 = it.nt * BN;
@@ -393,6 +430,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg<BN>::kTmemCols)
                  : "memory");
+  }
+  // the last CTA to finish re-arms the item counter for the next launch on this workspace
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const int done = atomicAdd(&g.status->sched_done, 1);
+    if (done == (int)gridDim.x - 1) {
+      g.status->sched_next = 0;
+      g.status->sched_done = 0;
+      __threadfence();
+    }
   }
 }
 
@@ -480,6 +527,7 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
   if (BN != 16 && BN != 64 && BN != 256) return TEMPLORA_ERR_INVALID_ARG;
   DeviceInfo *di = device_info();
   if (!di || di->cc_major != 10) return TEMPLORA_ERR_UNSUPPORTED;
+  if (!status) return TEMPLORA_ERR_WORKSPACE;  // the kernel keeps its item counter in the status record
 
   // heaviest work items first: the static round-robin schedule then ends on the short ones
   int order[kTcMaxProblems];

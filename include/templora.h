@@ -158,7 +158,8 @@ templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *c
 
 /*
  * Kernel-path selection for testing: 0 = automatic (tensor-core path when the
- * shape allows), 1 = always the generic kernel path.  Returns the previous value.
+ * shape allows, frozen-weight GEMMs on CTA pairs), 1 = always the generic kernel path,
+ * 2 = tensor-core path with single-CTA tiles only.  Returns the previous value.
  * Process-wide; not part of the method.
  */
 int32_t templora_set_kernel_path(int32_t mode);

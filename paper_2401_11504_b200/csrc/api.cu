@@ -75,6 +75,9 @@ bool use_tc(const templora_linear_t *lin, bool dry) {
   return dry ? true : tc_available();
 }
 
+// Frozen-weight GEMMs on CTA pairs unless kernel path 2 (single-CTA tensor-core tiles) is selected.
+int use_pairs() { return g_kernel_path.load() == 2 ? 0 : 1; }
+
 Operand op(const void *p, int dt, long long s0, long long s1) { return Operand{p, dt, s0, s1}; }
 
 // ---------------------------------------------------------------- problem builders (tensor-core path)
@@ -149,7 +152,7 @@ templora_status_t fwd_impl(const templora_linear_t *l, int T, const void *x, voi
     ReduceJob rj{Upart, su, Tr, Tr, l->s, 1.f, U_save, 0, Us};
     TL_TRY(reduce_partials_batch(&rj, 1, st));
     TcProblem py = prob_y(l, T, x, Us, y);
-    return tc_gemm_grouped(&py, 1, 256, ws.status(), st);
+    return tc_gemm_grouped(&py, 1, 256, ws.status(), st, use_pairs());
   }
   float *U = U_save ? U_save : ws.take<float>((size_t)Tr);
   if (dry) return TEMPLORA_OK;
@@ -198,7 +201,7 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
     TL_TRY(reduce_partials_batch(jobs, 2, st));
     if (dX) {
       TcProblem px = prob_dX(l, T, dY, Vs, dX);
-      TL_TRY(tc_gemm_grouped(&px, 1, 256, ws.status(), st));
+      TL_TRY(tc_gemm_grouped(&px, 1, 256, ws.status(), st, use_pairs()));
     }
     TcProblem grads[2] = {prob_dB(l, T, dY, Us, dBpart, sb), prob_dA(l, T, x, Vs, dApart, sa)};
     TL_TRY(tc_gemm_grouped(grads, 2, 64, ws.status(), st));
@@ -380,7 +383,7 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
     probs[np++] = prob_y(proj + i, T, x[i], b.Us[i], y[i]);
     if (dX && dX[i]) probs[np++] = prob_dX(proj + i, T, dY[i], b.Vs[i], dX[i]);
   }
-  TL_TRY(tc_gemm_grouped(probs, np, 256, status, st));
+  TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, use_pairs()));
   np = 0; nj = 0;
   for (int i = 0; i < n; ++i) {
     const templora_linear_t *l = proj + i;
@@ -622,7 +625,7 @@ templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *c
 }
 
 int32_t templora_set_kernel_path(int32_t mode) {
-  return g_kernel_path.exchange(mode == 1 ? 1 : 0);
+  return g_kernel_path.exchange((mode == 1 || mode == 2) ? mode : 0);
 }
 
 }  // extern "C"

@@ -116,8 +116,9 @@ struct TcProblem {
   long long out_split;        // element stride between split-K partial outputs
 };
 constexpr int kTcMaxProblems = 16;
-// BN: tile width, one of 16, 64, 256.
-templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st);
+// BN: tile width, one of 16, 64, 256.  cta_pairs != 0 with BN == 256 runs 256 x 256 tiles on CTA pairs.
+templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st,
+                                  int cta_pairs = 0);
 bool tc_available();
 
 // ---- workspace need of the decode-time forward alone (api.cu) -------------------

@@ -105,6 +105,13 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
   }
 }
 
+// Fast path of a wait: one poll inline, the bounded loop only when the barrier is not ready yet.
+__device__ __forceinline__ bool mbar_wait_fast(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                               DeviceStatus *st, int where) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait(bar, parity, abort_flag, st, where);
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -136,6 +143,14 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
   d |= 2ull << 61;  // 128-byte swizzle
   return d;
 }
+// Descriptor of an operand tile with the start-address field left zero, and the start-address step
+// (in 16-byte units) from one K = 16 slice to the next.  K-contiguous tiles advance 32 bytes inside
+// the 128-byte swizzled row; M/N-contiguous tiles advance two 8-row groups (2048 bytes).
+__device__ __forceinline__ uint64_t smem_desc_template(int mn_major) {
+  return mn_major ? smem_desc(0, 8192, 1024) : smem_desc(0, 16, 1024);
+}
+__device__ __forceinline__ uint32_t smem_desc_kstep(int mn_major) { return mn_major ? (2048u >> 4) : (32u >> 4); }
+
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N = n.
 __device__ __forceinline__ uint32_t instr_desc(int n, int a_mn, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
@@ -298,6 +313,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         const Item it = decode_item(g, item);
         const DevProb &q = g.p[it.p];
         const int n0 = it.nt * BN;
+        const int pa_mn = q.a_mn, pb_mn = q.b_mn;
         const int nmain = it.kb1 - it.kb0;
         const int nkb = nmain + it.next;
         for (int i = 0; i < nkb; ++i) {
@@ -305,16 +321,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
           const int kel = ext ? (i - nmain) * BK : (it.kb0 + i) * BK;
           const CUtensorMap *ma = ext ? &q.tmAe : &q.tmA;
           const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 100)) { ok = false; break; }
+          if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 100)) { ok = false; break; }
           mbar_arrive_expect_tx(full_bar(stage), kTxBytes);
           const uint32_t sA = smem0 + stage * kStage, sB = sA + kStageA;
-          if (!q.a_mn) {
+          if (!pa_mn) {
             tma_load_2d(sA, ma, full_bar(stage), kel, it.m0);
           } else {
 #pragma unroll
             for (int b = 0; b < BM / 64; ++b) tma_load_2d(sA + b * 8192, ma, full_bar(stage), it.m0 + b * 64, kel);
           }
-          if (!q.b_mn) {
+          if (!pb_mn) {
             tma_load_2d(sB, mb, full_bar(stage), kel, n0);
           } else {
 #pragma unroll
@@ -360,17 +376,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, g.status, 200)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        const uint32_t idesc = instr_desc(BN, q.a_mn, q.b_mn);
+        const int a_mn = q.a_mn, b_mn = q.b_mn;
+        const uint32_t idesc = instr_desc(BN, a_mn, b_mn);
+        const uint64_t a_tmpl = smem_desc_template(a_mn), b_tmpl = smem_desc_template(b_mn);
+        const uint32_t a_step = smem_desc_kstep(a_mn), b_step = smem_desc_kstep(b_mn);
         for (int i = 0; i < nkb; ++i) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, g.status, 201)) { ok = false; break; }
+          if (!mbar_wait_fast(full_bar(stage), phase, abort_flag, g.status, 201)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sA = smem0 + stage * kStage, sB = sA + kStageA;
+          const uint32_t a_lo = (smem0 + stage * kStage) >> 4, b_lo = a_lo + (kStageA >> 4);
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            const uint64_t ad = q.a_mn ? smem_desc(sA + kk * 2048, 8192, 1024) : smem_desc(sA + kk * 32, 16, 1024);
-            const uint64_t bd = q.b_mn ? smem_desc(sB + kk * 2048, 8192, 1024) : smem_desc(sB + kk * 32, 16, 1024);
-            tc_mma_bf16(d_tmem, ad, bd, idesc, (i | kk) != 0 ? 1u : 0u);
-          }
+          for (int kk = 0; kk < BK / 16; ++kk)
+            tc_mma_bf16(d_tmem, a_tmpl | (uint64_t)(a_lo + kk * a_step), b_tmpl | (uint64_t)(b_lo + kk * b_step), idesc,
+                        (i | kk) != 0 ? 1u : 0u);
           tc_commit(empty_bar(stage));  // frees the smem stage once these MMAs have read it
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -443,6 +460,257 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
   }
 }
 
+// ------------------------------------------------------------------ CTA-pair kernel (256 x 256 tiles)
+// Two CTAs of a cluster (one TPC) share one 256 x 256 output tile: each loads its own 128 rows of
+// the A operand and its own 128-column half of the B operand, and the even CTA issues
+// tcgen05.mma.cta_group::2 (M = 256), which reads both halves of B from the two CTAs' shared
+// memory.  Per flop this moves 1.5x fewer operand bytes from L2 into shared memory than 128 x 256
+// tiles on single CTAs, which is what bounds the frozen-weight GEMMs.  Each CTA drains its own
+// 128 x 256 half of the accumulator from its own TMEM.  Items are dealt round-robin to the pairs.
+namespace pair {
+
+constexpr int kStages = 6;
+constexpr int kStageB = 128 * BK * 2;            // this CTA's half of the B tile: 16 KB
+constexpr int kStage = kStageA + kStageB;        // 32 KB per CTA and stage
+constexpr int kSmemBytes = kStages * kStage + 1024 + 1024;
+constexpr int kTmemCols = 512;                   // two 256-column accumulators
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion is signalled on a barrier that may live in the peer CTA of the pair.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster, int c0,
+                                                 int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {  // arrives on `bar` in both CTAs of the pair
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t instr_desc_pair(int a_mn, int b_mn) {  // M = 256, N = 256
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+// item -> (problem, 256-row tile, 256-column tile); no split-K on this path
+__device__ __forceinline__ Item decode_item_pair(const DevGroup &g, int item) {
+  int p = 0;
+  while (p + 1 < g.n_prob && item >= g.p[p + 1].item_start) ++p;
+  const DevProb &q = g.p[p];
+  int local = item - q.item_start;
+  Item it;
+  it.p = p;
+  it.m0 = (local % q.m_tiles) * 256;
+  it.nt = local / q.m_tiles;
+  it.split = 0;
+  it.kb0 = 0;
+  it.kb1 = q.kb_main;
+  it.next = q.kb_ext;
+  return it;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+    tc_gemm_pair_kernel(const __grid_constant__ DevGroup g) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_al = smem_raw + (smem0 - smem_u32(smem_raw));
+  const uint32_t bar0 = smem0 + kStages * kStage;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };                        // used in the even CTA
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };           // one per CTA
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };       // one per CTA
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };  // used in the even CTA
+  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + kStages * kStage + 512);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 516);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();      // 0: issues the MMAs; 1: its peer
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);    // the even CTA's expect_tx covers the bytes of both CTAs
+      mbar_init(empty_bar(s), 1);   // one multicast commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);   // one multicast commit
+      mbar_init(tempty_bar(a), 8);  // four epilogue warps in each CTA
+    }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
+                 "r"((uint32_t)kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // the peer's barriers are initialised before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ===================== TMA producer (both CTAs) =====================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      long long issued = 0;
+      bool ok = true;
+      const uint32_t full0 = mapa_shared(full_bar(0), 0);
+      for (int item = pair_id; ok && item < g.n_items; item += n_pairs) {
+        const Item it = decode_item_pair(g, item);
+        const DevProb &q = g.p[it.p];
+        const int m0 = it.m0 + (int)rank * 128;          // this CTA's rows of the A operand
+        const int n0 = it.nt * 256 + (int)rank * 128;    // this CTA's half of the B operand
+        const int pa_mn = q.a_mn, pb_mn = q.b_mn;
+        const int nmain = it.kb1 - it.kb0;
+        const int nkb = nmain + it.next;
+        for (int i = 0; i < nkb; ++i) {
+          const bool ext = i >= nmain;
+          const int kel = ext ? (i - nmain) * BK : (it.kb0 + i) * BK;
+          const CUtensorMap *ma = ext ? &q.tmAe : &q.tmA;
+          const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
+          if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 400)) { ok = false; break; }
+          const uint32_t fb = full0 + 8u * stage;   // the even CTA's barrier
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2u * (uint32_t)kStage);
+          const uint32_t sA = smem0 + stage * kStage, sB = sA + kStageA;
+          if (!pa_mn) {
+            tma_load_2d_pair(sA, ma, fb, kel, m0);
+          } else {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sA + b * 8192, ma, fb, m0 + b * 64, kel);
+          }
+          if (!pb_mn) {
+            tma_load_2d_pair(sB, mb, fb, kel, n0);
+          } else {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sB + b * 8192, mb, fb, n0 + b * 64, kel);
+          }
+          ++issued;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok && rank == 0) {
+        long long n = issued < kStages ? issued : kStages;
+        for (long long k = 0; k < n; ++k) {
+          long long idx = issued - 1 - k;
+          int s = (int)(idx % kStages);
+          uint32_t ph = (uint32_t)((idx / kStages) & 1);
+          const unsigned long long t0 = globaltimer_ns();
+          while (!mbar_try(full_bar(s), ph) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer (even CTA only) =====================
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int item = pair_id; ok && item < g.n_items; item += n_pairs, ++local) {
+        const Item it = decode_item_pair(g, item);
+        const DevProb &q = g.p[it.p];
+        const int nkb = (it.kb1 - it.kb0) + it.next;
+        const int acc = local & 1;
+        const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, g.status, 500)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 256);
+        const int a_mn = q.a_mn, b_mn = q.b_mn;
+        const uint32_t idesc = instr_desc_pair(a_mn, b_mn);
+        const uint64_t a_tmpl = smem_desc_template(a_mn), b_tmpl = smem_desc_template(b_mn);
+        const uint32_t a_step = smem_desc_kstep(a_mn), b_step = smem_desc_kstep(b_mn);
+        for (int i = 0; i < nkb; ++i) {
+          if (!mbar_wait_fast(full_bar(stage), phase, abort_flag, g.status, 501)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_lo = (smem0 + stage * kStage) >> 4, b_lo = a_lo + (kStageA >> 4);
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk)
+            tc_mma_bf16_pair(d_tmem, a_tmpl | (uint64_t)(a_lo + kk * a_step), b_tmpl | (uint64_t)(b_lo + kk * b_step),
+                             idesc, (i | kk) != 0 ? 1u : 0u);
+          tc_commit_pair(empty_bar(stage));   // frees this stage in both CTAs
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit_pair(tfull_bar(acc));  // accumulator complete, both CTAs
+      }
+      if (!ok) {
+        tc_commit_pair(drain_bar);
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try(drain_bar, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ===================== epilogue (warps 2..5, both CTAs) =====================
+    const int quarter = warp & 3;
+    int local = 0;
+    bool ok = true;
+    for (int item = pair_id; ok && item < g.n_items; item += n_pairs, ++local) {
+      const Item it = decode_item_pair(g, item);
+      const DevProb &q = g.p[it.p];
+      const int n0 = it.nt * 256;
+      const int acc = local & 1;
+      const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, g.status, 600)) { ok = false; break; }
+      tc_fence_after();
+      const int row = it.m0 + (int)rank * 128 + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 256);
+      uint32_t v[32];
+#pragma unroll 1
+      for (int c0 = 0; c0 < 256; c0 += 32) {
+        tmem_ld32(t_row + c0, v);
+        tmem_ld_wait();
+        store_chunk<32>(q, v, row, n0 + c0, 0);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // neither CTA leaves while the other may still signal its barriers
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                 : "memory");
+  }
+}
+
+}  // namespace pair
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -484,6 +752,7 @@ struct DeviceInfo {
   int sm_count = 0;
   int cc_major = 0;
   bool attr_set[3] = {false, false, false};
+  bool pair_attr_set = false;
 };
 DeviceInfo *device_info() {
   static DeviceInfo info[64];
@@ -515,6 +784,22 @@ templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream
   return TEMPLORA_OK;
 }
 
+templora_status_t launch_pair(const DevGroup &g, DeviceInfo *di, cudaStream_t st) {
+  if (!di->pair_attr_set) {
+    TL_CUDA_CHECK(cudaFuncSetAttribute(pair::tc_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       pair::kSmemBytes));
+    di->pair_attr_set = true;
+  }
+  int pairs = di->sm_count / 2;
+  if (g.n_items < pairs) pairs = g.n_items;
+  {
+    LaunchScope scope(kKindTcMain, st);
+    pair::tc_gemm_pair_kernel<<<2 * pairs, kThreads, pair::kSmemBytes, st>>>(g);
+  }
+  TL_CUDA_CHECK(cudaGetLastError());
+  return TEMPLORA_OK;
+}
+
 }  // namespace
 
 bool tc_available() {
@@ -522,8 +807,12 @@ bool tc_available() {
   return di && di->cc_major == 10 && encode_fn() != nullptr;
 }
 
-templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st) {
+templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st,
+                                  int cta_pairs) {
   if (n <= 0 || n > kTcMaxProblems) return TEMPLORA_ERR_INVALID_ARG;
+  const bool use_pair = cta_pairs && BN == 256;   // 256 x 256 tiles on CTA pairs
+  const int tile_m = use_pair ? 256 : BM;         // rows of one work item
+  const int box_b = use_pair ? 128 : BN;          // rows of the B-operand box one CTA loads
   if (BN != 16 && BN != 64 && BN != 256) return TEMPLORA_ERR_INVALID_ARG;
   DeviceInfo *di = device_info();
   if (!di || di->cc_major != 10) return TEMPLORA_ERR_UNSUPPORTED;
@@ -557,7 +846,8 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     q.kb_main = (p.K + BK - 1) / BK;
     q.kb_ext = (p.Kext + BK - 1) / BK;
     q.splits = p.splits < 1 ? 1 : (p.splits > q.kb_main ? q.kb_main : p.splits);
-    q.m_tiles = (p.M + BM - 1) / BM;
+    if (use_pair && p.splits > 1) return TEMPLORA_ERR_UNSUPPORTED;
+    q.m_tiles = (p.M + tile_m - 1) / tile_m;
     q.n_tiles = (p.N + BN - 1) / BN;
     q.item_start = items;
     q.a_mn = p.a_mn; q.b_mn = p.b_mn;
@@ -567,11 +857,11 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     if (cnt + items > 0x3fffffff) return TEMPLORA_ERR_UNSUPPORTED;
     items += (int)cnt;
     bool ok = make_operand_map(&q.tmA, p.A, p.M, p.K, p.lda, p.a_mn, BM) &&
-              make_operand_map(&q.tmB, p.B, p.N, p.K, p.ldb, p.b_mn, BN);
+              make_operand_map(&q.tmB, p.B, p.N, p.K, p.ldb, p.b_mn, box_b);
     if (p.Kext > 0) {
       if (!p.Aext || !p.Bext || ((p.ldaext | p.ldbext) & 7)) return TEMPLORA_ERR_INVALID_ARG;
       ok = ok && make_operand_map(&q.tmAe, p.Aext, p.M, p.Kext, p.ldaext, p.a_mn, BM) &&
-           make_operand_map(&q.tmBe, p.Bext, p.N, p.Kext, p.ldbext, p.b_mn, BN);
+           make_operand_map(&q.tmBe, p.Bext, p.N, p.Kext, p.ldbext, p.b_mn, box_b);
     } else {
       q.tmAe = q.tmA;
       q.tmBe = q.tmB;
@@ -579,6 +869,7 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     if (!ok) return TEMPLORA_ERR_CUDA;
   }
   g.n_items = items;
+  if (use_pair) return launch_pair(g, di, st);
   if (BN == 256) return launch<256>(g, di, 0, st);
   if (BN == 64) return launch<64>(g, di, 1, st);
   return launch<16>(g, di, 2, st);

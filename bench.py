@@ -287,29 +287,38 @@ def decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=32, reps=5):
             lins.append(b.linear_desc(W0, A, B, s))
         blocks.append(lins)
     bytes_per_block = sum(inputs.decode_bytes(di, do, r) for _, di, do in projections)
-    ws_bytes = max(b.templora_workspace_bytes(l, 16) for l in blocks[0])
+    ws_bytes = max(max(b.templora_workspace_bytes(l, 16) for l in blocks[0]), b.templora_decode_block_workspace_bytes(blocks[0]))
     ws = b.alloc_workspace(ws_bytes, dev)
     out = {}
     for n in c["decode_tokens"]:
         xs = {di: inputs.make_tensor(0, "dec", f"x{n}-{di}", (n, di), "normal", 1.0, "bf16", dev) for di in (4096, 11008)}
         ys = {do: torch.empty((n, do), dtype=torch.bfloat16, device=dev) for do in (4096, 11008)}
 
-        def sweep():
+        def sweep_single():
             for lins in blocks:
                 for lin in lins:
                     b.templora_decode_fwd(lin, xs[lin.d_in], ys[lin.d_out], ws)
-        sweep()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
+
+        def sweep_block():
+            for a in block_args:
+                b.templora_decode_block_fwd(a, ws)
+
+        block_args = [b.DecodeBlockArgs(lins, [xs[l.d_in] for l in lins], [ys[l.d_out] for l in lins]) for lins in blocks]
+        res = {}
+        for label, sweep in (("per_projection_calls", sweep_single), ("one_call_per_block", sweep_block)):
             sweep()
-        e1.record()
-        torch.cuda.synchronize()
-        sec = e0.elapsed_time(e1) / 1e3 / (reps * n_blocks)
-        gbs = bytes_per_block / sec / 1e9
-        out[f"n{n}"] = {"us_per_block": sec * 1e6, "GBps": gbs, "frac_of_measured_hbm": gbs / peaks["hbm"],
-                        "frac_of_nominal_8000": gbs / 8000.0}
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                sweep()
+            e1.record()
+            torch.cuda.synchronize()
+            sec = e0.elapsed_time(e1) / 1e3 / (reps * n_blocks)
+            gbs = bytes_per_block / sec / 1e9
+            res[label] = {"us_per_block": sec * 1e6, "GBps": gbs, "frac_of_measured_hbm": gbs / peaks["hbm"],
+                          "frac_of_nominal_8000": gbs / 8000.0}
+        out[f"n{n}"] = res
     code, where = b.templora_read_device_status(ws)
     assert code == 0, f"decode device status {code} at {where}"
     out["bytes_per_block"] = bytes_per_block

@@ -127,6 +127,19 @@ templora_status_t templora_decode_fwd(const templora_linear_t *lin, int32_t n_to
                                       void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Decode-time forward of n_proj independent projections in one call (same formula and token
+ * limit as templora_decode_fwd).  Projections that do not depend on one another - q, k, v of
+ * one block, or gate and up - share launches: every W0 is still streamed exactly once, but
+ * the launch and pipeline ramp-up cost is paid once per group of up to 8 projections instead
+ * of once per projection.  proj, x, y are HOST arrays; x[i] [n_tokens, d_in_i] and
+ * y[i] [n_tokens, d_out_i] are device pointers.
+ */
+size_t templora_decode_block_workspace_bytes(const templora_linear_t *proj, int32_t n_proj);
+templora_status_t templora_decode_block_fwd(const templora_linear_t *proj, int32_t n_proj, int32_t n_tokens,
+                                            const void *const *x, void *const *y, void *ws, size_t ws_bytes,
+                                            void *stream);
+
+/*
  * The whole chunk update of n_proj projections: for each of `epochs` epochs, forward
  * and backward of every projection over the T-token chunk with the current A, B, then
  * one AdamW step on every A and B (batch = chunk, so one optimizer step per epoch;

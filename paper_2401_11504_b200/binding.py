@@ -21,6 +21,7 @@ EXPORTS = [
     "templora_linear_bwd", "templora_adamw_step", "templora_decode_fwd", "templora_update_block",
     "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
     "templora_timing_enable", "templora_timing_read", "templora_decode_fwd_noalloc",
+    "templora_decode_block_workspace_bytes", "templora_decode_block_fwd",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH = range(7)
@@ -71,6 +72,10 @@ def _load():
     lib.templora_read_device_status.argtypes = [vp, vp, C.POINTER(i32), C.POINTER(i32)]
     lib.templora_set_kernel_path.restype = i32
     lib.templora_set_kernel_path.argtypes = [i32]
+    lib.templora_decode_block_workspace_bytes.restype = sz
+    lib.templora_decode_block_workspace_bytes.argtypes = [LP, i32]
+    lib.templora_decode_block_fwd.restype = i32
+    lib.templora_decode_block_fwd.argtypes = [LP, i32, i32, C.POINTER(vp), C.POINTER(vp), vp, sz, vp]
     lib.templora_decode_fwd_noalloc.restype = i32
     lib.templora_decode_fwd_noalloc.argtypes = [LP, i32, vp, vp, vp]
     lib.templora_timing_enable.restype = None
@@ -225,3 +230,25 @@ def templora_decode_fwd_noalloc(lin, x, y, stream=None):
     all calls on the device, so calls that could overlap on the GPU must be serialised."""
     _check(lib.templora_decode_fwd_noalloc(C.byref(lin), x.shape[0], _ptr(x), _ptr(y), _stream(stream)),
            "templora_decode_fwd_noalloc")
+
+
+def templora_decode_block_workspace_bytes(lins):
+    arr = (LinearDesc * len(lins))(*lins)
+    return int(lib.templora_decode_block_workspace_bytes(arr, len(lins)))
+
+
+class DecodeBlockArgs:
+    """Marshalled argument arrays of templora_decode_block_fwd, built once and reusable."""
+
+    def __init__(self, lins, xs, ys):
+        n = len(lins)
+        self.n, self.n_tokens = n, xs[0].shape[0]
+        self.lins = (LinearDesc * n)(*lins)
+        self.x = (C.c_void_p * n)(*[t.data_ptr() for t in xs])
+        self.y = (C.c_void_p * n)(*[t.data_ptr() for t in ys])
+        self._keep = (lins, xs, ys)
+
+
+def templora_decode_block_fwd(args, ws, stream=None):
+    _check(lib.templora_decode_block_fwd(args.lins, args.n, args.n_tokens, args.x, args.y, _ptr(ws), ws.numel(),
+                                         _stream(stream)), "templora_decode_block_fwd")

@@ -260,81 +260,180 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
 }
 
 // ---------------------------------------------------------------- decode
-// y[i,o] = sum_k P[k][i][o] + s * sum_j (sum_k Pu[k][i][j]) * B[o][j]     (rank-r term added in registers)
+// Finish of the decode-time forward, for up to kDecGroup projections in one launch:
+//   y[i,o] = sum_k P[k][i][o] + s * sum_j (sum_k Pu[k][i][j]) * B[o][j]
+// P, Pu are the split-K partial slabs of W0 x^T and A x^T written by the tensor-core kernel; the
+// rank-r term is added in registers.  One thread per output feature o, all n tokens.
 constexpr int kFinThreads = 128;
-__global__ void __launch_bounds__(kFinThreads) decode_finish_kernel(const float *__restrict__ P, int sp,
-                                                                    const float *__restrict__ Pu, int spu, int n,
-                                                                    int d_out, int r, float s,
-                                                                    const __nv_bfloat16 *__restrict__ B,
-                                                                    __nv_bfloat16 *__restrict__ y) {
-  extern __shared__ float u_sm[];  // [n][r], already scaled by s
-  for (int e = threadIdx.x; e < n * r; e += kFinThreads) {
-    float a = 0.f;
-    for (int k = 0; k < spu; ++k) a += Pu[(long long)k * n * r + e];
-    u_sm[e] = s * a;
-  }
-  __syncthreads();
-  const int o = blockIdx.x * kFinThreads + threadIdx.x;
-  if (o >= d_out) return;
-  float acc[16];
+constexpr int kDecGroup = 8;
+struct FinishEntry {
+  const float *P, *Pu;
+  const __nv_bfloat16 *B;
+  __nv_bfloat16 *y;
+  int sp, spu, d_out, r, block_start;
+  float s;
+};
+struct FinishBatch {
+  FinishEntry e[kDecGroup];
+  int n_entries, n_tokens;
+};
+
+template <int N>
+__device__ __forceinline__ void finish_body(const FinishEntry &f, int o, const float *u_sm, int ru) {
+  float acc[N];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    acc[i] = 0.f;
-    if (i < n)
-      for (int k = 0; k < sp; ++k) acc[i] += P[((long long)k * n + i) * d_out + o];
+  for (int i = 0; i < N; ++i) {
+    float a = 0.f;
+    for (int k = 0; k < f.sp; ++k) a += f.P[((long long)k * N + i) * f.d_out + o];
+    acc[i] = a;
   }
-  const __nv_bfloat16 *brow = B + (long long)o * r;
-  for (int j0 = 0; j0 < r; j0 += 8) {  // r is a multiple of 8 on this path
-    uint4 w = *reinterpret_cast<const uint4 *>(brow + j0);
+  const __nv_bfloat16 *brow = f.B + (long long)o * f.r;
+  for (int j0 = 0; j0 < f.r; j0 += 8) {  // r is a multiple of 8 on this path
+    const uint4 w = *reinterpret_cast<const uint4 *>(brow + j0);
     const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&w);
     float b[8];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      float2 f = __bfloat1622float2(h[e]);
-      b[2 * e] = f.x; b[2 * e + 1] = f.y;
+      const float2 t = __bfloat1622float2(h[e]);
+      b[2 * e] = t.x; b[2 * e + 1] = t.y;
     }
 #pragma unroll
-    for (int i = 0; i < 16; ++i)
-      if (i < n) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[i] = fmaf(u_sm[i * r + j0 + e], b[e], acc[i]);
-      }
+    for (int i = 0; i < N; ++i) {
+      const float4 u0 = *reinterpret_cast<const float4 *>(u_sm + i * ru + j0);       // broadcast reads
+      const float4 u1 = *reinterpret_cast<const float4 *>(u_sm + i * ru + j0 + 4);
+      float a = acc[i];
+      a = fmaf(u0.x, b[0], a); a = fmaf(u0.y, b[1], a); a = fmaf(u0.z, b[2], a); a = fmaf(u0.w, b[3], a);
+      a = fmaf(u1.x, b[4], a); a = fmaf(u1.y, b[5], a); a = fmaf(u1.z, b[6], a); a = fmaf(u1.w, b[7], a);
+      acc[i] = a;
+    }
   }
 #pragma unroll
-  for (int i = 0; i < 16; ++i)
-    if (i < n) y[(long long)i * d_out + o] = __float2bfloat16_rn(acc[i]);
+  for (int i = 0; i < N; ++i) f.y[(long long)i * f.d_out + o] = __float2bfloat16_rn(acc[i]);
+}
+
+__global__ void __launch_bounds__(kFinThreads) decode_finish_kernel(const __grid_constant__ FinishBatch fb) {
+  __shared__ __align__(16) float u_sm[16 * 256];  // [n][r] (r <= 256), already scaled by s
+  int j = 0;
+  while (j + 1 < fb.n_entries && (int)blockIdx.x >= fb.e[j + 1].block_start) ++j;
+  const FinishEntry &f = fb.e[j];
+  const int n = fb.n_tokens;
+  for (int e = threadIdx.x; e < n * f.r; e += kFinThreads) {
+    float a = 0.f;
+    for (int k = 0; k < f.spu; ++k) a += f.Pu[(long long)k * n * f.r + e];
+    u_sm[e] = f.s * a;
+  }
+  __syncthreads();
+  const int o = (blockIdx.x - f.block_start) * kFinThreads + threadIdx.x;
+  if (o >= f.d_out) return;
+  switch (n) {   // token count fixed at compile time so that the accumulators stay in registers
+    case 1: finish_body<1>(f, o, u_sm, f.r); break;
+    case 2: finish_body<2>(f, o, u_sm, f.r); break;
+    case 3: finish_body<3>(f, o, u_sm, f.r); break;
+    case 4: finish_body<4>(f, o, u_sm, f.r); break;
+    case 5: finish_body<5>(f, o, u_sm, f.r); break;
+    case 6: finish_body<6>(f, o, u_sm, f.r); break;
+    case 7: finish_body<7>(f, o, u_sm, f.r); break;
+    case 8: finish_body<8>(f, o, u_sm, f.r); break;
+    case 9: finish_body<9>(f, o, u_sm, f.r); break;
+    case 10: finish_body<10>(f, o, u_sm, f.r); break;
+    case 11: finish_body<11>(f, o, u_sm, f.r); break;
+    case 12: finish_body<12>(f, o, u_sm, f.r); break;
+    case 13: finish_body<13>(f, o, u_sm, f.r); break;
+    case 14: finish_body<14>(f, o, u_sm, f.r); break;
+    case 15: finish_body<15>(f, o, u_sm, f.r); break;
+    default: finish_body<16>(f, o, u_sm, f.r); break;
+  }
+}
+
+// Split-K factor of the decode stream of one projection launched together with others whose
+// k-blocks add up to total_kb.  Few tokens: about 12 work items per SM (short tail, the partial
+// slabs are tiny); many tokens: about 6 (the slabs grow with the token count).  Never fewer than
+// 8 k-blocks per item.
+int decode_splits(int kb, long long total_kb, int n) {
+  const int per_sm = n <= 4 ? 12 : 6;
+  long long target = (total_kb + kSmRef * per_sm - 1) / (kSmRef * per_sm);
+  if (target < 8) target = 8;
+  long long s = (kb + target / 2) / target;
+  if (s < 1) s = 1;
+  if (s > 16) s = 16;
+  if (s > kb) s = kb;
+  return (int)s;
+}
+// Rows of partial sums to reserve per output feature so that any token count 1..16 fits.
+int decode_partial_rows(int kb, long long total_kb) {
+  const int a = decode_splits(kb, total_kb, 4) * 4, b = decode_splits(kb, total_kb, 16) * 16;
+  return a > b ? a : b;
+}
+
+// Decode-time forward of up to kDecGroup projections (all on the tensor-core path): one grouped
+// launch streams every W0 and A once, one launch finishes.
+templora_status_t decode_group_tc(const templora_linear_t *proj, int np, int n, const void *const *x, void *const *y,
+                                  WsAlloc &ws, bool dry, cudaStream_t st) {
+  long long total_kb = 0;
+  for (int i = 0; i < np; ++i)
+    total_kb += (long long)(cdiv(proj[i].d_out, 128) + cdiv(proj[i].r, 128)) * cdiv(proj[i].d_in, 64);
+  TcProblem p[2 * kDecGroup] = {};
+  FinishBatch fb;
+  fb.n_entries = np; fb.n_tokens = n;
+  int blocks = 0;
+  for (int i = 0; i < np; ++i) {
+    const templora_linear_t *l = proj + i;
+    const int kb = cdiv(l->d_in, 64);
+    const int sp = decode_splits(kb, total_kb, n), spu = sp;
+    const int rows = decode_partial_rows(kb, total_kb);
+    float *P = ws.take<float>((size_t)rows * l->d_out);
+    float *Pu = ws.take<float>((size_t)rows * l->r);
+    if (dry) continue;
+    if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+    TcProblem &a = p[2 * i], &u = p[2 * i + 1];
+    a.M = l->d_out; a.N = n; a.K = l->d_in;
+    a.A = l->W0; a.lda = l->d_in; a.B = x[i]; a.ldb = l->d_in;
+    a.splits = sp; a.out = P; a.out_f32 = 1; a.out_s0 = 1; a.out_s1 = l->d_out; a.out_split = (long long)n * l->d_out;
+    u.M = l->r; u.N = n; u.K = l->d_in;
+    u.A = l->A; u.lda = l->d_in; u.B = x[i]; u.ldb = l->d_in;
+    u.splits = spu; u.out = Pu; u.out_f32 = 1; u.out_s0 = 1; u.out_s1 = l->r; u.out_split = (long long)n * l->r;
+    fb.e[i] = FinishEntry{P, Pu, reinterpret_cast<const __nv_bfloat16 *>(l->B), reinterpret_cast<__nv_bfloat16 *>(y[i]),
+                          sp, spu, l->d_out, l->r, blocks, l->s};
+    blocks += cdiv(l->d_out, kFinThreads);
+  }
+  if (dry) return TEMPLORA_OK;
+  TL_TRY(tc_gemm_grouped(p, 2 * np, 16, ws.status(), st));
+  {
+    LaunchScope scope(kKindDecodeFinish, st);
+    decode_finish_kernel<<<blocks, kFinThreads, 0, st>>>(fb);
+  }
+  TL_CUDA_CHECK(cudaGetLastError());
+  return TEMPLORA_OK;
 }
 
 templora_status_t decode_impl(const templora_linear_t *l, int n, const void *x, void *y, WsAlloc &ws, bool dry,
                               cudaStream_t st) {
-  if (use_tc(l, dry)) {
-    const int kb = cdiv(l->d_in, 64);
-    const int sp = pick_splits(cdiv(l->d_out, 128), kb, 1);
-    const int spu = pick_splits(cdiv(l->r, 128), kb, 1);
-    float *P = ws.take<float>((size_t)sp * 16 * l->d_out);
-    float *Pu = ws.take<float>((size_t)spu * 16 * l->r);
-    if (dry) return TEMPLORA_OK;
-    if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
-    TcProblem p[2] = {};
-    p[0].M = l->d_out; p[0].N = n; p[0].K = l->d_in;
-    p[0].A = l->W0; p[0].lda = l->d_in; p[0].B = x; p[0].ldb = l->d_in;
-    p[0].splits = sp; p[0].out = P; p[0].out_f32 = 1; p[0].out_s0 = 1; p[0].out_s1 = l->d_out;
-    p[0].out_split = (long long)n * l->d_out;
-    p[1].M = l->r; p[1].N = n; p[1].K = l->d_in;
-    p[1].A = l->A; p[1].lda = l->d_in; p[1].B = x; p[1].ldb = l->d_in;
-    p[1].splits = spu; p[1].out = Pu; p[1].out_f32 = 1; p[1].out_s0 = 1; p[1].out_s1 = l->r;
-    p[1].out_split = (long long)n * l->r;
-    TL_TRY(tc_gemm_grouped(p, 2, 16, ws.status(), st));
-    {
-      LaunchScope scope(kKindDecodeFinish, st);
-      decode_finish_kernel<<<cdiv(l->d_out, kFinThreads), kFinThreads, (size_t)n * l->r * sizeof(float), st>>>(
-          P, sp, Pu, spu, n, l->d_out, l->r, l->s, reinterpret_cast<const __nv_bfloat16 *>(l->B),
-          reinterpret_cast<__nv_bfloat16 *>(y));
-    }
-    TL_CUDA_CHECK(cudaGetLastError());
-    return TEMPLORA_OK;
-  }
+  if (use_tc(l, dry)) return decode_group_tc(l, 1, n, &x, &y, ws, dry, st);
   return fwd_impl(l, n, x, y, nullptr, ws, dry, st);
+}
+
+// Several independent projections in one call.  Groups of kDecGroup run one after another on the
+// stream and reuse the same workspace region.
+templora_status_t decode_block_impl(const templora_linear_t *proj, int n_proj, int n, const void *const *x,
+                                    void *const *y, void *ws_ptr, size_t ws_bytes, bool dry, size_t *need,
+                                    cudaStream_t st) {
+  size_t max_need = kStatusBytes;
+  int i = 0;
+  while (i < n_proj) {
+    WsAlloc a(dry ? nullptr : ws_ptr, ws_bytes);
+    if (use_tc(proj + i, dry)) {
+      int np = 1;
+      while (i + np < n_proj && np < kDecGroup && use_tc(proj + i + np, dry)) ++np;
+      TL_TRY(decode_group_tc(proj + i, np, n, dry ? nullptr : x + i, dry ? nullptr : y + i, a, dry, st));
+      i += np;
+    } else {
+      TL_TRY(fwd_impl(proj + i, n, dry ? nullptr : x[i], dry ? nullptr : y[i], nullptr, a, dry, st));
+      i += 1;
+    }
+    if (a.off > max_need) max_need = a.off;
+  }
+  if (need) *need = max_need;
+  return TEMPLORA_OK;
 }
 
 // ---------------------------------------------------------------- update_block (tensor-core, grouped)
@@ -570,6 +669,37 @@ templora_status_t templora_decode_fwd(const templora_linear_t *lin, int32_t n_to
   TL_TRY(check_ws(ws, ws_bytes));
   WsAlloc a(ws, ws_bytes);
   return decode_impl(lin, n_tokens, x, y, a, false, reinterpret_cast<cudaStream_t>(stream));
+}
+
+size_t templora_decode_block_workspace_bytes(const templora_linear_t *proj, int32_t n_proj) {
+  if (!proj || n_proj <= 0) return 0;
+  for (int i = 0; i < n_proj; ++i)
+    if (check_linear(proj + i) != TEMPLORA_OK) return 0;
+  size_t need = 0, best = kStatusBytes;
+  for (int mode = 0; mode < 2; ++mode) {
+    t_path_override = mode;
+    decode_block_impl(proj, n_proj, 16, nullptr, nullptr, nullptr, 0, true, &need, nullptr);
+    if (need > best) best = need;
+  }
+  t_path_override = -1;
+  return best;
+}
+
+templora_status_t templora_decode_block_fwd(const templora_linear_t *proj, int32_t n_proj, int32_t n_tokens,
+                                            const void *const *x, void *const *y, void *ws, size_t ws_bytes,
+                                            void *stream) {
+  if (!proj || n_proj <= 0 || !x || !y || n_tokens < 1 || n_tokens > 16) return TEMPLORA_ERR_INVALID_ARG;
+  for (int i = 0; i < n_proj; ++i) {
+    TL_TRY(check_linear(proj + i));
+    TL_TRY(check_linear_ptrs(proj + i));
+    if (!x[i] || !y[i] || !aligned16(x[i]) || !aligned16(y[i])) return TEMPLORA_ERR_INVALID_ARG;
+  }
+  TL_TRY(check_ws(ws, ws_bytes));
+  size_t need = 0;
+  decode_block_impl(proj, n_proj, n_tokens, nullptr, nullptr, nullptr, 0, true, &need, nullptr);
+  if (ws_bytes < need) return TEMPLORA_ERR_WORKSPACE;
+  return decode_block_impl(proj, n_proj, n_tokens, x, y, ws, ws_bytes, false, nullptr,
+                           reinterpret_cast<cudaStream_t>(stream));
 }
 
 templora_status_t templora_update_block(const templora_linear_t *proj, const templora_param_t *A_state,

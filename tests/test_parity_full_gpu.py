@@ -126,3 +126,26 @@ def test_config3_decode_7b_block(b, n):
             assert b.templora_read_device_status(ws)[0] == 0
             ref = orc.decode_fwd(f64(x), f64(W0), f64(A), f64(B), c["s"])
             assert_close(f"{tag} decode n={n}", f64(y), ref, TOL["bf16"])
+
+
+@pytest.mark.parametrize("n", inputs.CONFIGS[3]["decode_tokens"])
+def test_config3_decode_whole_block_in_one_call(b, n):
+    # the launch configuration the benchmark times for decode: the seven projections of a block
+    # through templora_decode_block_fwd
+    c = inputs.CONFIGS[3]
+    lins, xs, ys, keep = [], [], [], []
+    for name, d_in, d_out in c["projections"]:
+        tag = f"cfg3b/{name}"
+        W0 = inputs.make_tensor(0, tag, "W0", (d_out, d_in), "normal", d_in ** -0.5, "bf16", "cuda")
+        A = inputs.make_tensor(0, tag, "A", (c["r"], d_in), "uniform", d_in ** -0.5, "bf16", "cuda")
+        B = inputs.make_tensor(0, tag, "B", (d_out, c["r"]), "normal", 0.02, "bf16", "cuda")
+        xs.append(inputs.make_tensor(0, tag, f"x{n}", (n, d_in), "normal", 1.0, "bf16", "cuda"))
+        ys.append(torch.full((n, d_out), float("nan"), dtype=torch.bfloat16, device="cuda"))
+        lins.append(b.linear_desc(W0, A, B, c["s"]))
+        keep.append((W0, A, B))
+    ws = b.alloc_workspace(b.templora_decode_block_workspace_bytes(lins))
+    b.templora_decode_block_fwd(b.DecodeBlockArgs(lins, xs, ys), ws)
+    assert b.templora_read_device_status(ws)[0] == 0
+    for (W0, A, B), x, y in zip(keep, xs, ys):
+        ref = orc.decode_fwd(f64(x), f64(W0), f64(A), f64(B), c["s"])
+        assert_close(f"decode block n={n}", f64(y), ref, TOL["bf16"])

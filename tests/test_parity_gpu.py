@@ -117,6 +117,34 @@ def test_decode_fp32_and_generic(generic_path):
         assert_close("decode y", f64(y), ref, TOL[dtype])
 
 
+def test_decode_block_matches_oracle(b):
+    # eleven independent projections in one call: more than one group of eight, mixed shapes,
+    # one of them (d_in = 100) outside the tensor-core path
+    shapes = [(512, 640, 64), (512, 640, 64), (1024, 264, 16), (2048, 512, 64), (100, 60, 4)] * 2 + [(4096, 1024, 64)]
+    for n in (1, 5, 16):
+        hosts = [inputs.make_linear(14, f"decblk-{n}-{i}", n, di, do, r, dtype="bf16") for i, (di, do, r) in enumerate(shapes)]
+        devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
+        lins = [b.linear_desc(d["W0"], d["A"], d["B"], 2.0) for d in devs]
+        ys = [torch.full((n, do), float("nan"), dtype=torch.bfloat16, device="cuda") for _, do, _ in shapes]
+        ws = b.alloc_workspace(b.templora_decode_block_workspace_bytes(lins))
+        args = b.DecodeBlockArgs(lins, [d["x"] for d in devs], ys)
+        b.templora_decode_block_fwd(args, ws)
+        assert b.templora_read_device_status(ws)[0] == 0
+        for i, h in enumerate(hosts):
+            ref = orc.decode_fwd(f64(h["x"]), f64(h["W0"]), f64(h["A"]), f64(h["B"]), 2.0)
+            assert_close(f"decode block y{i} n={n}", f64(ys[i]), ref, TOL["bf16"])
+
+
+def test_single_cta_tensor_core_path(b):
+    # kernel path 2: frozen-weight GEMMs on single-CTA 128 x 256 tiles instead of CTA pairs
+    b.templora_set_kernel_path(2)
+    try:
+        check_fwd_bwd(b, 15, "tc-single", 300, 328, 520, 24, 2.0, "bf16")
+        check_fwd_bwd(b, 15, "tc-single2", 640, 1024, 768, 64, 2.0, "bf16")
+    finally:
+        b.templora_set_kernel_path(0)
+
+
 # ------------------------------------------------------------------ AdamW
 def _adamw_case(b, n, dtype, steps, hp, seed):
     hp = hp32(hp)

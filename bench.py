@@ -318,6 +318,18 @@ def decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=32, reps=5):
             gbs = bytes_per_block / sec / 1e9
             res[label] = {"us_per_block": sec * 1e6, "GBps": gbs, "frac_of_measured_hbm": gbs / peaks["hbm"],
                           "frac_of_nominal_8000": gbs / 8000.0}
+        # where the time of the one-call-per-block mode goes: device time per kernel class
+        for k in (b.KIND_TC_DECODE, b.KIND_DECODE_FINISH):
+            b.templora_timing_read(k, reset=True)
+        b.templora_timing_enable(True)
+        sweep_block()
+        torch.cuda.synchronize()
+        b.templora_timing_enable(False)
+        ms_tc, n_tc, _ = b.templora_timing_read(b.KIND_TC_DECODE, reset=True)
+        ms_fin, n_fin, _ = b.templora_timing_read(b.KIND_DECODE_FINISH, reset=True)
+        res["one_call_per_block"]["stream_kernel_us"] = 1e3 * ms_tc / max(n_tc, 1)
+        res["one_call_per_block"]["finish_kernel_us"] = 1e3 * ms_fin / max(n_fin, 1)
+        res["one_call_per_block"]["stream_kernel_GBps"] = bytes_per_block / (ms_tc / max(n_tc, 1) * 1e-3) / 1e9
         out[f"n{n}"] = res
     code, where = b.templora_read_device_status(ws)
     assert code == 0, f"decode device status {code} at {where}"

@@ -263,8 +263,7 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
 // Finish of the decode-time forward, for up to kDecGroup projections in one launch:
 //   y[i,o] = sum_k P[k][i][o] + s * sum_j (sum_k Pu[k][i][j]) * B[o][j]
 // P, Pu are the split-K partial slabs of W0 x^T and A x^T written by the tensor-core kernel; the
-// rank-r term is added in registers.  One thread per output feature o, all n tokens.
-constexpr int kFinThreads = 128;
+// rank-r term is added in registers.
 constexpr int kDecGroup = 8;
 struct FinishEntry {
   const float *P, *Pu;
@@ -278,70 +277,56 @@ struct FinishBatch {
   int n_entries, n_tokens;
 };
 
-template <int N>
-__device__ __forceinline__ void finish_body(const FinishEntry &f, int o, const float *u_sm, int ru) {
-  float acc[N];
-#pragma unroll
-  for (int i = 0; i < N; ++i) {
-    float a = 0.f;
-    for (int k = 0; k < f.sp; ++k) a += f.P[((long long)k * N + i) * f.d_out + o];
-    acc[i] = a;
-  }
-  const __nv_bfloat16 *brow = f.B + (long long)o * f.r;
-  for (int j0 = 0; j0 < f.r; j0 += 8) {  // r is a multiple of 8 on this path
-    const uint4 w = *reinterpret_cast<const uint4 *>(brow + j0);
-    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&w);
-    float b[8];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float2 t = __bfloat1622float2(h[e]);
-      b[2 * e] = t.x; b[2 * e + 1] = t.y;
-    }
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-      const float4 u0 = *reinterpret_cast<const float4 *>(u_sm + i * ru + j0);       // broadcast reads
-      const float4 u1 = *reinterpret_cast<const float4 *>(u_sm + i * ru + j0 + 4);
-      float a = acc[i];
-      a = fmaf(u0.x, b[0], a); a = fmaf(u0.y, b[1], a); a = fmaf(u0.z, b[2], a); a = fmaf(u0.w, b[3], a);
-      a = fmaf(u1.x, b[4], a); a = fmaf(u1.y, b[5], a); a = fmaf(u1.z, b[6], a); a = fmaf(u1.w, b[7], a);
-      acc[i] = a;
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < N; ++i) f.y[(long long)i * f.d_out + o] = __float2bfloat16_rn(acc[i]);
-}
+// Block = kFinO output features x TY token lanes.  The block first stages its kFinO rows of B in
+// shared memory with coalesced loads (row pitch padded by 16 bytes: conflict-free row-per-thread
+// reads) and the scaled u = s * (A x^T) of all tokens; then thread (o, ty) finishes tokens ty, ty+TY, ...
+constexpr int kFinO = 64;
+constexpr int kFinTy = 4;   // 256 threads per block: the whole grid (d_out / 64 blocks) is resident at once
 
-__global__ void __launch_bounds__(kFinThreads) decode_finish_kernel(const __grid_constant__ FinishBatch fb) {
-  __shared__ __align__(16) float u_sm[16 * 256];  // [n][r] (r <= 256), already scaled by s
+__global__ void __launch_bounds__(kFinO * kFinTy, 6) decode_finish_kernel(const __grid_constant__ FinishBatch fb) {
+  extern __shared__ __align__(16) uint8_t fin_smem[];
   int j = 0;
   while (j + 1 < fb.n_entries && (int)blockIdx.x >= fb.e[j + 1].block_start) ++j;
   const FinishEntry &f = fb.e[j];
-  const int n = fb.n_tokens;
-  for (int e = threadIdx.x; e < n * f.r; e += kFinThreads) {
+  const int n = fb.n_tokens, r = f.r, d_out = f.d_out;
+  const int pitch = r + 8;                                        // bf16 elements per staged row of B
+  __nv_bfloat16 *b_sm = reinterpret_cast<__nv_bfloat16 *>(fin_smem);
+  float *u_sm = reinterpret_cast<float *>(fin_smem + (size_t)kFinO * pitch * 2);   // [n][r]
+  const int tid = threadIdx.y * kFinO + threadIdx.x, nthreads = kFinO * blockDim.y;
+  const int o0 = (blockIdx.x - f.block_start) * kFinO;
+
+  // stage B[o0 .. o0+kFinO) x r (16-byte chunks, coalesced along r)
+  const int chunks_per_row = r >> 3;
+  for (int c = tid; c < kFinO * chunks_per_row; c += nthreads) {
+    const int row = c / chunks_per_row, ch = c - row * chunks_per_row;
+    uint4 w = make_uint4(0, 0, 0, 0);
+    if (o0 + row < d_out) w = *reinterpret_cast<const uint4 *>(f.B + (long long)(o0 + row) * r + ch * 8);
+    *reinterpret_cast<uint4 *>(b_sm + row * pitch + ch * 8) = w;
+  }
+  for (int e = tid; e < n * r; e += nthreads) {
     float a = 0.f;
-    for (int k = 0; k < f.spu; ++k) a += f.Pu[(long long)k * n * f.r + e];
+    for (int k = 0; k < f.spu; ++k) a += f.Pu[(long long)k * n * r + e];
     u_sm[e] = f.s * a;
   }
   __syncthreads();
-  const int o = (blockIdx.x - f.block_start) * kFinThreads + threadIdx.x;
-  if (o >= f.d_out) return;
-  switch (n) {   // token count fixed at compile time so that the accumulators stay in registers
-    case 1: finish_body<1>(f, o, u_sm, f.r); break;
-    case 2: finish_body<2>(f, o, u_sm, f.r); break;
-    case 3: finish_body<3>(f, o, u_sm, f.r); break;
-    case 4: finish_body<4>(f, o, u_sm, f.r); break;
-    case 5: finish_body<5>(f, o, u_sm, f.r); break;
-    case 6: finish_body<6>(f, o, u_sm, f.r); break;
-    case 7: finish_body<7>(f, o, u_sm, f.r); break;
-    case 8: finish_body<8>(f, o, u_sm, f.r); break;
-    case 9: finish_body<9>(f, o, u_sm, f.r); break;
-    case 10: finish_body<10>(f, o, u_sm, f.r); break;
-    case 11: finish_body<11>(f, o, u_sm, f.r); break;
-    case 12: finish_body<12>(f, o, u_sm, f.r); break;
-    case 13: finish_body<13>(f, o, u_sm, f.r); break;
-    case 14: finish_body<14>(f, o, u_sm, f.r); break;
-    case 15: finish_body<15>(f, o, u_sm, f.r); break;
-    default: finish_body<16>(f, o, u_sm, f.r); break;
+  const int o = o0 + threadIdx.x;
+  if (o >= d_out) return;
+  const __nv_bfloat16 *brow = b_sm + threadIdx.x * pitch;
+  for (int i = threadIdx.y; i < n; i += blockDim.y) {
+    float acc = 0.f;
+    for (int k = 0; k < f.sp; ++k) acc += f.P[((long long)k * n + i) * d_out + o];
+    const float *urow = u_sm + i * r;
+    for (int j0 = 0; j0 < r; j0 += 8) {
+      const uint4 w = *reinterpret_cast<const uint4 *>(brow + j0);
+      const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&w);
+      const float4 u0 = *reinterpret_cast<const float4 *>(urow + j0);       // same address across the warp
+      const float4 u1 = *reinterpret_cast<const float4 *>(urow + j0 + 4);
+      const float2 b0 = __bfloat1622float2(h[0]), b1 = __bfloat1622float2(h[1]);
+      const float2 b2 = __bfloat1622float2(h[2]), b3 = __bfloat1622float2(h[3]);
+      acc = fmaf(u0.x, b0.x, acc); acc = fmaf(u0.y, b0.y, acc); acc = fmaf(u0.z, b1.x, acc); acc = fmaf(u0.w, b1.y, acc);
+      acc = fmaf(u1.x, b2.x, acc); acc = fmaf(u1.y, b2.y, acc); acc = fmaf(u1.z, b3.x, acc); acc = fmaf(u1.w, b3.y, acc);
+    }
+    f.y[(long long)i * d_out + o] = __float2bfloat16_rn(acc);
   }
 }
 
@@ -375,7 +360,7 @@ templora_status_t decode_group_tc(const templora_linear_t *proj, int np, int n, 
   TcProblem p[2 * kDecGroup] = {};
   FinishBatch fb;
   fb.n_entries = np; fb.n_tokens = n;
-  int blocks = 0;
+  int blocks = 0, max_r = 0;
   for (int i = 0; i < np; ++i) {
     const templora_linear_t *l = proj + i;
     const int kb = cdiv(l->d_in, 64);
@@ -394,13 +379,24 @@ templora_status_t decode_group_tc(const templora_linear_t *proj, int np, int n, 
     u.splits = spu; u.out = Pu; u.out_f32 = 1; u.out_s0 = 1; u.out_s1 = l->r; u.out_split = (long long)n * l->r;
     fb.e[i] = FinishEntry{P, Pu, reinterpret_cast<const __nv_bfloat16 *>(l->B), reinterpret_cast<__nv_bfloat16 *>(y[i]),
                           sp, spu, l->d_out, l->r, blocks, l->s};
-    blocks += cdiv(l->d_out, kFinThreads);
+    blocks += cdiv(l->d_out, kFinO);
+    if (l->r > max_r) max_r = l->r;
   }
   if (dry) return TEMPLORA_OK;
   TL_TRY(tc_gemm_grouped(p, 2 * np, 16, ws.status(), st));
   {
     LaunchScope scope(kKindDecodeFinish, st);
-    decode_finish_kernel<<<blocks, kFinThreads, 0, st>>>(fb);
+    const size_t smem = (size_t)kFinO * (max_r + 8) * 2 + (size_t)n * max_r * sizeof(float);
+    static bool attr_done_dev[64] = {};   // function attributes are per device
+    int dev_id = 0;
+    TL_CUDA_CHECK(cudaGetDevice(&dev_id));
+    bool &attr_done = attr_done_dev[dev_id & 63];
+    if (!attr_done) {
+      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50));
+      attr_done = true;
+    }
+    decode_finish_kernel<<<blocks, dim3(kFinO, kFinTy), smem, st>>>(fb);
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;

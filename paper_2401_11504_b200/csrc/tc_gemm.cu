@@ -31,16 +31,19 @@ constexpr int kSched = 4;  // depth of the work-item ring between the producer a
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 constexpr int kStageA = BM * BK * 2;  // 16 KB
-template <int BN, int STAGES, int TMEM_COLS> struct CfgBase {
-  static constexpr int kStages = STAGES, kTmemCols = TMEM_COLS;
+// KPS = k-blocks per pipeline stage.  The decode stream (BN = 16) moves two k-blocks per stage so that
+// the two 128-byte pieces of every W0 row are requested back to back (256 contiguous bytes per row).
+template <int BN, int STAGES, int TMEM_COLS, int KPS> struct CfgBase {
+  static constexpr int kStages = STAGES, kTmemCols = TMEM_COLS, kKps = KPS;
   static constexpr int kStageB = BN * BK * 2;
-  static constexpr int kStage = kStageA + kStageB;
+  static constexpr int kSub = kStageA + kStageB;       // one k-block of A and B
+  static constexpr int kStage = KPS * kSub;
   static constexpr int kSmemBytes = STAGES * kStage + 1024 /*barriers*/ + 1024 /*alignment slack*/;
 };
 template <int BN> struct Cfg;
-template <> struct Cfg<256> : CfgBase<256, 4, 512> {};
-template <> struct Cfg<64> : CfgBase<64, 8, 128> {};
-template <> struct Cfg<16> : CfgBase<16, 10, 32> {};
+template <> struct Cfg<256> : CfgBase<256, 4, 512, 1> {};
+template <> struct Cfg<64> : CfgBase<64, 8, 128, 1> {};
+template <> struct Cfg<16> : CfgBase<16, 3, 32, 4> {};
 
 struct alignas(64) DevProb {
   CUtensorMap tmA, tmB, tmAe, tmBe;
@@ -244,7 +247,8 @@ template <int BN>
 __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ DevGroup g) {
   constexpr int kStages = Cfg<BN>::kStages;
   constexpr int kStage = Cfg<BN>::kStage;
-  constexpr uint32_t kTxBytes = (uint32_t)kStage;
+  constexpr int kSub = Cfg<BN>::kSub;
+  constexpr int kKps = Cfg<BN>::kKps;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -316,26 +320,30 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         const int pa_mn = q.a_mn, pb_mn = q.b_mn;
         const int nmain = it.kb1 - it.kb0;
         const int nkb = nmain + it.next;
-        for (int i = 0; i < nkb; ++i) {
-          const bool ext = i >= nmain;
-          const int kel = ext ? (i - nmain) * BK : (it.kb0 + i) * BK;
-          const CUtensorMap *ma = ext ? &q.tmAe : &q.tmA;
-          const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
+        for (int i0 = 0; i0 < nkb; i0 += kKps) {
+          const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
           if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 100)) { ok = false; break; }
-          mbar_arrive_expect_tx(full_bar(stage), kTxBytes);
-          const uint32_t sA = smem0 + stage * kStage, sB = sA + kStageA;
-          if (!pa_mn) {
-            tma_load_2d(sA, ma, full_bar(stage), kel, it.m0);
-          } else {
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(cnt * kSub));
+          for (int j = 0; j < cnt; ++j) {
+            const int i = i0 + j;
+            const bool ext = i >= nmain;
+            const int kel = ext ? (i - nmain) * BK : (it.kb0 + i) * BK;
+            const CUtensorMap *ma = ext ? &q.tmAe : &q.tmA;
+            const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
+            const uint32_t sA = smem0 + stage * kStage + j * kSub, sB = sA + kStageA;
+            if (!pa_mn) {
+              tma_load_2d(sA, ma, full_bar(stage), kel, it.m0);
+            } else {
 #pragma unroll
-            for (int b = 0; b < BM / 64; ++b) tma_load_2d(sA + b * 8192, ma, full_bar(stage), it.m0 + b * 64, kel);
-          }
-          if (!pb_mn) {
-            tma_load_2d(sB, mb, full_bar(stage), kel, n0);
-          } else {
+              for (int b = 0; b < BM / 64; ++b) tma_load_2d(sA + b * 8192, ma, full_bar(stage), it.m0 + b * 64, kel);
+            }
+            if (!pb_mn) {
+              tma_load_2d(sB, mb, full_bar(stage), kel, n0);
+            } else {
 #pragma unroll
-            for (int b = 0; b < (BN >= 64 ? BN / 64 : 1); ++b)
-              tma_load_2d(sB + b * 8192, mb, full_bar(stage), n0 + b * 64, kel);
+              for (int b = 0; b < (BN >= 64 ? BN / 64 : 1); ++b)
+                tma_load_2d(sB + b * 8192, mb, full_bar(stage), n0 + b * 64, kel);
+            }
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -380,14 +388,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         const uint32_t idesc = instr_desc(BN, a_mn, b_mn);
         const uint64_t a_tmpl = smem_desc_template(a_mn), b_tmpl = smem_desc_template(b_mn);
         const uint32_t a_step = smem_desc_kstep(a_mn), b_step = smem_desc_kstep(b_mn);
-        for (int i = 0; i < nkb; ++i) {
+        for (int i0 = 0; i0 < nkb; i0 += kKps) {
+          const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
           if (!mbar_wait_fast(full_bar(stage), phase, abort_flag, g.status, 201)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_lo = (smem0 + stage * kStage) >> 4, b_lo = a_lo + (kStageA >> 4);
+          for (int j = 0; j < cnt; ++j) {
+            const uint32_t a_lo = (smem0 + stage * kStage + j * kSub) >> 4, b_lo = a_lo + (kStageA >> 4);
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk)
-            tc_mma_bf16(d_tmem, a_tmpl | (uint64_t)(a_lo + kk * a_step), b_tmpl | (uint64_t)(b_lo + kk * b_step), idesc,
-                        (i | kk) != 0 ? 1u : 0u);
+            for (int kk = 0; kk < BK / 16; ++kk)
+              tc_mma_bf16(d_tmem, a_tmpl | (uint64_t)(a_lo + kk * a_step), b_tmpl | (uint64_t)(b_lo + kk * b_step),
+                          idesc, (i0 | j | kk) != 0 ? 1u : 0u);
+          }
           tc_commit(empty_bar(stage));  // frees the smem stage once these MMAs have read it
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }

@@ -91,7 +91,7 @@ def test_bf16_unaligned_shape_takes_generic_path_automatically(b):
 
 # ------------------------------------------------------------------ decode
 @pytest.mark.parametrize("n", [1, 4, 16, 7])
-@pytest.mark.parametrize("d_in,d_out,r", [(512, 640, 64), (4096, 1024, 64), (1000, 264, 16)])
+@pytest.mark.parametrize("d_in,d_out,r", [(512, 640, 64), (4096, 1024, 64), (1000, 264, 16), (512, 384, 128), (256, 136, 256)])
 def test_decode_matches_oracle(b, n, d_in, d_out, r):
     host = inputs.make_linear(9, f"dec-{n}-{d_in}-{d_out}", n, d_in, d_out, r, dtype="bf16")
     dev = {k: v.cuda() for k, v in host.items()}

@@ -205,13 +205,14 @@ templora_status_t templora_decode_fwd_noalloc(const templora_linear_t *lin, int3
 
 /*
  * Launch accounting, a profiling aid (the paper has no counterpart).  The library counts
- * the launches of each kernel class; with timing enabled it also records a pair of CUDA
- * events on the launching stream around every launch.  Kernel classes: 0 tensor-core GEMM
+ * the launches of each kernel class; for the classes selected by kind_mask (bit k = class k,
+ * -1 = all, 0 = none) it also records a pair of CUDA events on the launching stream around
+ * every launch (which costs the timed kernel and its successor their early scheduling).  Kernel classes: 0 tensor-core GEMM
  * with 256-wide tiles (y, dX), 1 tensor-core GEMM with 64-wide tiles (U, V, dA, dB),
  * 2 tensor-core GEMM with 16-wide tiles (decode), 3 partial reduction, 4 AdamW,
  * 5 generic GEMM, 6 decode finish.  Process-wide.
  */
-void templora_timing_enable(int32_t on);
+void templora_timing_enable(int32_t kind_mask);
 
 /*
  * Waits for the recorded events of class `kind` and returns their summed device time

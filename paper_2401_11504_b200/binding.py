@@ -212,8 +212,17 @@ def templora_set_kernel_path(mode):
     return int(lib.templora_set_kernel_path(int(mode)))
 
 
-def templora_timing_enable(on):
-    lib.templora_timing_enable(int(bool(on)))
+def templora_timing_enable(kinds):
+    """kinds: iterable of kernel classes to time, True for all, False/None for none."""
+    if kinds is True:
+        mask = -1
+    elif not kinds:
+        mask = 0
+    else:
+        mask = 0
+        for k in kinds:
+            mask |= 1 << int(k)
+    lib.templora_timing_enable(mask)
 
 
 def templora_timing_read(kind, reset=False):

@@ -285,6 +285,7 @@ constexpr int kFinTy = 4;   // 256 threads per block: the whole grid (d_out / 64
 
 __global__ void __launch_bounds__(kFinO * kFinTy, 6) decode_finish_kernel(const __grid_constant__ FinishBatch fb) {
   extern __shared__ __align__(16) uint8_t fin_smem[];
+  pdl_prologue();
   int j = 0;
   while (j + 1 < fb.n_entries && (int)blockIdx.x >= fb.e[j + 1].block_start) ++j;
   const FinishEntry &f = fb.e[j];
@@ -396,7 +397,7 @@ templora_status_t decode_group_tc(const templora_linear_t *proj, int np, int n, 
       TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50));
       attr_done = true;
     }
-    decode_finish_kernel<<<blocks, dim3(kFinO, kFinTy), smem, st>>>(fb);
+    TL_CUDA_CHECK(launch_pdl(decode_finish_kernel, dim3(blocks), dim3(kFinO, kFinTy), smem, st, fb));
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <utility>
 
 #include "templora.h"
 
@@ -60,6 +61,33 @@ class LaunchScope {
   cudaStream_t st_;
   cudaEvent_t a_, b_;
 };
+
+// ---- programmatic dependent launch ----------------------------------------------
+// Every kernel of the library starts with pdl_prologue(): it waits until the kernels before it on
+// the stream have completed and flushed (so ordering is exactly that of plain stream launches)
+// and then lets the kernel after it be scheduled early, which hides that kernel's launch latency
+// behind this one's execution.  launch_pdl() launches with that attribute set.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
 
 // ---- generic (SIMT) GEMM:  D = alpha1 * A1 B1 + alpha2 * A2 B2 (+ D) --------
 // Element (i,k) of an operand lives at p[i*s0 + k*s1]; dt is a templora_dtype_t.

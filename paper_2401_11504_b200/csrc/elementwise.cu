@@ -16,6 +16,7 @@ constexpr int kRedThreads = 256;
 constexpr int kRedPerBlock = kRedThreads * 4;
 
 __global__ void __launch_bounds__(kRedThreads) reduce_partials_kernel(const __grid_constant__ ReduceBatch b) {
+  pdl_prologue();
   int j = 0;
   while (j + 1 < b.n_jobs && (int)blockIdx.x >= b.block_start[j + 1]) ++j;
   const ReduceJob &jb = b.job[j];
@@ -73,6 +74,7 @@ __device__ __forceinline__ void adam_one(float &p, float &m, float &v, float g, 
 }
 
 __global__ void __launch_bounds__(kAdamThreads) adamw_kernel(const __grid_constant__ AdamBatch b) {
+  pdl_prologue();
   int j = 0;
   while (j + 1 < b.n_tensors && (int)blockIdx.x >= b.block_start[j + 1]) ++j;
   const AdamTensor &t = b.t[j];
@@ -130,7 +132,7 @@ templora_status_t reduce_partials_batch(const ReduceJob *jobs, int n_jobs, cudaS
     b.block_start[b.n_jobs] = blocks;
     {
       LaunchScope scope(kKindReduce, st);
-      reduce_partials_kernel<<<blocks, kRedThreads, 0, st>>>(b);
+      TL_CUDA_CHECK(launch_pdl(reduce_partials_kernel, dim3(blocks), dim3(kRedThreads), 0, st, b));
     }
     TL_CUDA_CHECK(cudaGetLastError());
   }
@@ -164,7 +166,7 @@ templora_status_t adamw_launch(const templora_param_t *params, int n_params, flo
     b.block_start[b.n_tensors] = (int)blocks;
     {
       LaunchScope scope(kKindAdamW, st);
-      adamw_kernel<<<(unsigned)blocks, kAdamThreads, 0, st>>>(b);
+      TL_CUDA_CHECK(launch_pdl(adamw_kernel, dim3((unsigned)blocks), dim3(kAdamThreads), 0, st, b));
     }
     TL_CUDA_CHECK(cudaGetLastError());
   }

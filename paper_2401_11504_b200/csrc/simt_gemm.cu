@@ -56,6 +56,7 @@ __device__ __forceinline__ void product(const Operand &A, const Operand &B, int 
 __global__ void __launch_bounds__(NT) simt_gemm_kernel(const SimtGemm g) {
   __shared__ float sA[TK][TM + 1];
   __shared__ float sB[TK][TN + 1];
+  pdl_prologue();
   const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
   const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
 
@@ -92,7 +93,7 @@ templora_status_t simt_gemm(const SimtGemm &g, cudaStream_t st) {
   if (grid.y > 65535u) return TEMPLORA_ERR_UNSUPPORTED;
   {
     LaunchScope scope(kKindSimt, st);
-    simt_gemm_kernel<<<grid, NT, 0, st>>>(g);
+    TL_CUDA_CHECK(launch_pdl(simt_gemm_kernel, grid, dim3(NT), 0, st, g));
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;

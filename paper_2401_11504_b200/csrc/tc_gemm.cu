@@ -297,6 +297,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_prologue();   // the set-up above touched no global memory and may overlap the previous kernel's tail
 
   if (warp == 0) {
     // ===================== TMA producer =====================
@@ -590,6 +591,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
   cluster_sync_all();   // the peer's barriers are initialised before anything is sent to them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_prologue();   // the set-up above touched no global memory and may overlap the previous kernel's tail
 
   if (warp == 0) {
     // ===================== TMA producer (both CTAs) =====================
@@ -789,7 +791,7 @@ templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream
   int grid = g.n_items < di->sm_count ? g.n_items : di->sm_count;
   {
     LaunchScope scope(BN == 256 ? kKindTcMain : (BN == 64 ? kKindTcSkinny : kKindTcDecode), st);
-    tc_gemm_kernel<BN><<<grid, kThreads, Cfg<BN>::kSmemBytes, st>>>(g);
+    TL_CUDA_CHECK(launch_pdl(tc_gemm_kernel<BN>, dim3(grid), dim3(kThreads), Cfg<BN>::kSmemBytes, st, g));
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;
@@ -805,7 +807,7 @@ templora_status_t launch_pair(const DevGroup &g, DeviceInfo *di, cudaStream_t st
   if (g.n_items < pairs) pairs = g.n_items;
   {
     LaunchScope scope(kKindTcMain, st);
-    pair::tc_gemm_pair_kernel<<<2 * pairs, kThreads, pair::kSmemBytes, st>>>(g);
+    TL_CUDA_CHECK(launch_pdl(pair::tc_gemm_pair_kernel, dim3(2 * pairs), dim3(kThreads), pair::kSmemBytes, st, g));
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;

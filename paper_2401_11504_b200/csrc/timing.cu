@@ -21,7 +21,7 @@ std::vector<Pair> g_free;
 
 LaunchScope::LaunchScope(int kind, cudaStream_t st) : kind_(kind), st_(st), a_(nullptr), b_(nullptr) {
   g_launches[kind].fetch_add(1, std::memory_order_relaxed);
-  if (!g_timing_on.load(std::memory_order_relaxed)) return;
+  if (!((g_timing_on.load(std::memory_order_relaxed) >> kind) & 1)) return;
   std::lock_guard<std::mutex> lk(g_mu);
   Pair p{nullptr, nullptr};
   if (!g_free.empty()) {
@@ -47,7 +47,7 @@ using namespace templora;
 
 extern "C" {
 
-void templora_timing_enable(int32_t on) { g_timing_on.store(on ? 1 : 0); }
+void templora_timing_enable(int32_t kind_mask) { g_timing_on.store(kind_mask); }
 
 templora_status_t templora_timing_read(int32_t kind, double *total_ms, int64_t *timed_launches, int64_t *all_launches,
                                        int32_t reset) {

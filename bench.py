@@ -229,35 +229,57 @@ def run_ours(args):
         kernel_share[name] = round(ms / max(share_ms, 1e-9), 4)
 
     # ---- end to end: host buffers in, updated module out, copies inside the timed region ----
+    # Every step copies that step's x and dY from pinned host memory to the device, runs the chunk
+    # update and copies the updated bf16 A and B back.  The device input buffers are double-buffered:
+    # the copy of step i+1 runs on a second stream while step i computes (what a serving loop does).
     blk = blocks[0]
-    host_in = [(torch.empty_like(t, device="cpu").pin_memory().copy_(t), t) for t in blk.x + blk.dY]
+    ins0 = blk.x + blk.dY
+    ins1 = [torch.empty_like(t) for t in ins0]
+    n_x = len(blk.x)
+    args_e2e = [blk.args, b.UpdateBlockArgs(blk.lins, blk.A_desc, blk.B_desc, ins1[:n_x], ins1[n_x:], blk.y, blk.dX)]
+    dev_in = [ins0, ins1]
+    host_in = [torch.empty_like(t, device="cpu").pin_memory().copy_(t) for t in ins0]
     outs = [st[nm]["work"] for st in blk.state for nm in ("A", "B")]
     host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in outs]
-    h2d = sum(h.numel() * h.element_size() for h, _ in host_in)
+    h2d = sum(h.numel() * h.element_size() for h in host_in)
     d2h = sum(h.numel() * h.element_size() for h in host_out)
+    copy_stream = torch.cuda.Stream(device=dev)
+    ready = [torch.cuda.Event(), torch.cuda.Event()]     # inputs of buffer set k have landed
+    consumed = [torch.cuda.Event(), torch.cuda.Event()]  # the update that read buffer set k is done
 
-    def e2e_step():
-        for h, d in host_in:
-            d.copy_(h, non_blocking=True)
-        steps_taken[0] = b.templora_update_block(blk.args, 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
-                                                 hp["weight_decay"], steps_taken[0], ws)
-        for h, d in zip(host_out, outs):
-            h.copy_(d, non_blocking=True)
+    def upload(i):
+        k = i % 2
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(consumed[k])
+            for h, d in zip(host_in, dev_in[k]):
+                d.copy_(h, non_blocking=True)
+            ready[k].record(copy_stream)
+
+    def e2e_run(n_steps):
+        for k in range(2):
+            consumed[k].record(stream)
+        upload(0)
+        for i in range(n_steps):
+            k = i % 2
+            if i + 1 < n_steps:
+                upload(i + 1)
+            stream.wait_event(ready[k])
+            steps_taken[0] = b.templora_update_block(args_e2e[k], 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                                     hp["weight_decay"], steps_taken[0], ws)
+            consumed[k].record(stream)
+            for h, d in zip(host_out, outs):
+                h.copy_(d, non_blocking=True)
         torch.cuda.synchronize()
 
-    for _ in range(3):
-        e2e_step()
+    e2e_run(3)
     n_e2e = max(3, min(args.steps, 30))
     ranks.barrier()
-    t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(n_e2e):
-        e2e_step()
-    e1.record(stream)
     torch.cuda.synchronize()
-    e2e_seconds = max(e0.elapsed_time(e1) / 1e3, time.perf_counter() - t0)
-    e2e_value, _ = runtime.aggregate_throughput(T * n_e2e, e2e_seconds, ranks)
+    t0 = time.perf_counter()
+    e2e_run(n_e2e)
+    e2e_seconds = time.perf_counter() - t0     # host clock around fully synchronised work: covers both streams
+    e2e_seconds = ranks.max_over_ranks(e2e_seconds)
+    e2e_value = ranks.sum_over_ranks(T * n_e2e) / e2e_seconds
 
     # ---- decode-time LoRA GEMV bandwidth (second figure of the metric) -------
     decode = None
@@ -278,7 +300,7 @@ def run_ours(args):
                            "step_tflops": tf_block, "step_frac_of_measured_sustained": tf_block / ranks.world / peaks["tflops"],
                            "step_frac_of_nominal_2250": tf_block / ranks.world / 2250.0},
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                        "steps": n_e2e, "what": "x and dY of the 7 projections from pinned host memory in; updated bf16 A and B out"},
+                        "steps": n_e2e, "what": "per step: x and dY of the 7 projections from pinned host memory in (double-buffered, copy of step i+1 overlaps compute of step i), updated bf16 A and B out"},
                 "gpu_launches": int(launches), "roofline": roofline, "kernel_time_share": kernel_share,
                 "clocks": clk.summary(), "cpu_baseline": cpu, "decode": decode}
         print(json.dumps(line))

@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel (bytes), from an ncu capture summarised under
 # profiles/; valid only while the kernel source is the one that was profiled.
-TRAFFIC = {"tc_gemm_sha1": "f154ec92815dd38f8c38bd02f02292b8c775504a", "bytes_per_launch": 1232277272}
+TRAFFIC = {"tc_gemm_sha1": "f70d89e890faacd7f68bfa15e4540389bf707b4d", "bytes_per_launch": 1248943872}
 
 
 def load_peaks():

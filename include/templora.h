@@ -159,6 +159,20 @@ templora_status_t templora_update_block(const templora_linear_t *proj, const tem
                                         float eps, float weight_decay, int64_t *step_inout,
                                         void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * The same update with the chunk cut into batches of batch_tokens rows (the last may be
+ * shorter): forward, backward and one AdamW step per batch, so each epoch takes
+ * ceil(T / batch_tokens) optimizer steps (the paper's cost table: chunk 2048, batch 1024,
+ * 2 epochs = 4 steps).  batch_tokens >= T is templora_update_block.  Gradient buffers hold
+ * the last batch's gradients on return.
+ */
+templora_status_t templora_update_block_batched(const templora_linear_t *proj, const templora_param_t *A_state,
+                                                const templora_param_t *B_state, int32_t n_proj, int32_t T,
+                                                int32_t batch_tokens, const void *const *x, const void *const *dY,
+                                                void *const *y, void *const *dX, int32_t epochs, float lr,
+                                                float beta1, float beta2, float eps, float weight_decay,
+                                                int64_t *step_inout, void *ws, size_t ws_bytes, void *stream);
+
 /* Static description of a status code. */
 const char *templora_status_string(templora_status_t st);
 

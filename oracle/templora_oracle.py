@@ -116,13 +116,16 @@ def round_bf16(a):
 # the whole update of one block of projections: n epochs over the chunk,
 # one optimizer step per epoch (batch = chunk)
 # --------------------------------------------------------------------------
-def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf16_work=False):
+def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf16_work=False, batch=None):
     """projs: list of dicts with keys x, dY, W0, s, A_master, B_master and optionally
     mA, vA, mB, vB (default 0).  For each epoch: forward and backward of every
     projection with the current working A, B; then step += 1 and AdamW on every
     A and B.  With bf16_work the GEMMs read round_bf16(master), the optimizer
     updates the master (fp32 master + bf16 working copy, which is what bfloat16
-    training under ZeRO-2 implies).
+    training under ZeRO-2 implies).  With batch < T every epoch walks the chunk in
+    row slices of `batch` tokens and takes one optimizer step per slice (the cost
+    table's "training steps" = epochs * chunk / batch); y and dX are then filled
+    slice by slice and dA, dB are the last slice's.
 
     Returns (state, step): state[i] has A_master, B_master, mA, vA, mB, vB and the
     last epoch's y, dX, dA, dB.
@@ -135,16 +138,24 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
                        mA=_f64(p.get("mA", np.zeros_like(A))), vA=_f64(p.get("vA", np.zeros_like(A))),
                        mB=_f64(p.get("mB", np.zeros_like(B))), vB=_f64(p.get("vB", np.zeros_like(B)))))
     step = int(step0)
+    T = np.asarray(projs[0]["x"]).shape[0]
+    batch = T if batch is None or batch >= T else int(batch)
+    for p, q in zip(projs, st):
+        q["y"] = np.zeros((T, np.asarray(p["W0"]).shape[0]), dtype=F64)
+        q["dX"] = np.zeros((T, np.asarray(p["W0"]).shape[1]), dtype=F64)
     for _ in range(int(epochs)):
-        for p, q in zip(projs, st):
-            A = round_bf16(q["A_master"]) if bf16_work else q["A_master"]
-            B = round_bf16(q["B_master"]) if bf16_work else q["B_master"]
-            q["y"], _ = linear_fwd(p["x"], p["W0"], A, B, p["s"])
-            q["dX"], q["dA"], q["dB"] = linear_bwd(p["x"], p["dY"], p["W0"], A, B, p["s"])
-        step += 1
-        for q in st:
-            q["A_master"], q["mA"], q["vA"] = adamw_step(q["A_master"], q["dA"], q["mA"], q["vA"],
-                                                         lr, beta1, beta2, eps, weight_decay, step)
-            q["B_master"], q["mB"], q["vB"] = adamw_step(q["B_master"], q["dB"], q["mB"], q["vB"],
-                                                         lr, beta1, beta2, eps, weight_decay, step)
+        for r0 in range(0, T, batch):
+            rows = slice(r0, min(r0 + batch, T))
+            for p, q in zip(projs, st):
+                A = round_bf16(q["A_master"]) if bf16_work else q["A_master"]
+                B = round_bf16(q["B_master"]) if bf16_work else q["B_master"]
+                xb, dYb = _f64(p["x"])[rows], _f64(p["dY"])[rows]
+                q["y"][rows], _ = linear_fwd(xb, p["W0"], A, B, p["s"])
+                q["dX"][rows], q["dA"], q["dB"] = linear_bwd(xb, dYb, p["W0"], A, B, p["s"])
+            step += 1
+            for q in st:
+                q["A_master"], q["mA"], q["vA"] = adamw_step(q["A_master"], q["dA"], q["mA"], q["vA"],
+                                                             lr, beta1, beta2, eps, weight_decay, step)
+                q["B_master"], q["mB"], q["vB"] = adamw_step(q["B_master"], q["dB"], q["mB"], q["vB"],
+                                                             lr, beta1, beta2, eps, weight_decay, step)
     return st, step

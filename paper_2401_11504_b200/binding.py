@@ -21,7 +21,7 @@ EXPORTS = [
     "templora_linear_bwd", "templora_adamw_step", "templora_decode_fwd", "templora_update_block",
     "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
     "templora_timing_enable", "templora_timing_read", "templora_decode_fwd_noalloc",
-    "templora_decode_block_workspace_bytes", "templora_decode_block_fwd",
+    "templora_decode_block_workspace_bytes", "templora_decode_block_fwd", "templora_update_block_batched",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH = range(7)
@@ -66,6 +66,9 @@ def _load():
     lib.templora_update_block.restype = i32
     lib.templora_update_block.argtypes = [LP, PP, PP, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                           C.POINTER(vp), i32, f32, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_update_block_batched.restype = i32
+    lib.templora_update_block_batched.argtypes = [LP, PP, PP, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                                  C.POINTER(vp), i32, f32, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
     lib.templora_status_string.restype = C.c_char_p
     lib.templora_status_string.argtypes = [i32]
     lib.templora_read_device_status.restype = i32
@@ -198,6 +201,17 @@ def templora_update_block(args, epochs, lr, beta1, beta2, eps, weight_decay, ste
     _check(lib.templora_update_block(args.lins, args.A, args.B, args.n, args.T, args.x, args.dY, args.y, args.dX,
                                      int(epochs), lr, beta1, beta2, eps, weight_decay, C.byref(st), _ptr(ws),
                                      ws.numel(), _stream(stream)), "templora_update_block")
+    return st.value
+
+
+def templora_update_block_batched(args, batch_tokens, epochs, lr, beta1, beta2, eps, weight_decay, step, ws,
+                                  stream=None):
+    """Chunk update with one optimizer step per batch of batch_tokens rows; returns the new step count."""
+    st = C.c_int64(int(step))
+    _check(lib.templora_update_block_batched(args.lins, args.A, args.B, args.n, args.T, int(batch_tokens), args.x,
+                                             args.dY, args.y, args.dX, int(epochs), lr, beta1, beta2, eps,
+                                             weight_decay, C.byref(st), _ptr(ws), ws.numel(), _stream(stream)),
+           "templora_update_block_batched")
     return st.value
 
 

@@ -495,11 +495,14 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
   return TEMPLORA_OK;
 }
 
+// One epoch = the chunk's T rows in slices of `batch` rows (the last may be shorter), one optimizer
+// step after each slice: epochs * ceil(T / batch) steps in all.
 templora_status_t update_impl(const templora_linear_t *proj, const templora_param_t *As, const templora_param_t *Bs,
-                              int n_proj, int T, const void *const *x, const void *const *dY, void *const *y,
-                              void *const *dX, int epochs, float lr, float b1, float b2, float eps, float wd,
-                              int64_t *step_inout, void *ws_ptr, size_t ws_bytes, bool dry, size_t *need,
-                              cudaStream_t st) {
+                              int n_proj, int T_chunk, int batch, const void *const *x_chunk,
+                              const void *const *dY_chunk, void *const *y_chunk, void *const *dX_chunk, int epochs,
+                              float lr, float b1, float b2, float eps, float wd, int64_t *step_inout, void *ws_ptr,
+                              size_t ws_bytes, bool dry, size_t *need, cudaStream_t st) {
+  const int T = (batch <= 0 || batch > T_chunk) ? T_chunk : batch;   // rows of a full slice
   bool all_tc = true;
   for (int i = 0; i < n_proj; ++i) all_tc = all_tc && use_tc(proj + i, dry);
   // workspace: the largest need of any group (groups run one after another on the stream)
@@ -529,24 +532,40 @@ templora_status_t update_impl(const templora_linear_t *proj, const templora_para
   all.reserve(2 * (size_t)n_proj);
   for (int i = 0; i < n_proj; ++i) { all.push_back(As[i]); all.push_back(Bs[i]); }
   const int work_bf16 = proj[0].dtype == TEMPLORA_BF16;
+  const size_t esize = work_bf16 ? 2 : 4;
+  std::vector<const void *> xs(n_proj), dYs(n_proj);
+  std::vector<void *> ys(n_proj), dXs(n_proj);
   int64_t step = *step_inout;
-  for (int e = 0; e < epochs; ++e) {
+  for (int e = 0; e < epochs; ++e)
+   for (int r0 = 0; r0 < T_chunk; r0 += T) {
+    const int rows = (T_chunk - r0 < T) ? T_chunk - r0 : T;
+    for (int i = 0; i < n_proj; ++i) {
+      const size_t oi = (size_t)r0 * proj[i].d_in * esize, oo = (size_t)r0 * proj[i].d_out * esize;
+      xs[i] = reinterpret_cast<const uint8_t *>(x_chunk[i]) + oi;
+      dYs[i] = reinterpret_cast<const uint8_t *>(dY_chunk[i]) + oo;
+      ys[i] = reinterpret_cast<uint8_t *>(y_chunk[i]) + oo;
+      dXs[i] = (dX_chunk && dX_chunk[i]) ? reinterpret_cast<uint8_t *>(dX_chunk[i]) + oi : nullptr;
+    }
+    const void *const *x = xs.data();
+    const void *const *dY = dYs.data();
+    void *const *y = ys.data();
+    void *const *dX = dX_chunk ? dXs.data() : nullptr;
     if (all_tc) {
       for (int g0 = 0; g0 < n_proj; g0 += kGroup) {
         const int n = (n_proj - g0 < kGroup) ? n_proj - g0 : kGroup;
         WsAlloc a(ws_ptr, ws_bytes);
         GroupBufs gb;
-        carve_group(proj + g0, n, T, a, gb);
+        carve_group(proj + g0, n, rows, a, gb);
         if (a.overflow) return TEMPLORA_ERR_WORKSPACE;
-        TL_TRY(update_group_tc(proj + g0, As + g0, Bs + g0, n, T, x + g0, dY + g0, y + g0, dX ? dX + g0 : nullptr, gb,
-                               a.status(), st));
+        TL_TRY(update_group_tc(proj + g0, As + g0, Bs + g0, n, rows, x + g0, dY + g0, y + g0, dX ? dX + g0 : nullptr,
+                               gb, a.status(), st));
       }
     } else {
       for (int i = 0; i < n_proj; ++i) {
         WsAlloc a(ws_ptr, ws_bytes);
-        TL_TRY(fwd_impl(proj + i, T, x[i], y[i], nullptr, a, false, st));
+        TL_TRY(fwd_impl(proj + i, rows, x[i], y[i], nullptr, a, false, st));
         WsAlloc c(ws_ptr, ws_bytes);
-        TL_TRY(bwd_impl(proj + i, T, x[i], dY[i], nullptr, dX ? dX[i] : nullptr, const_cast<float *>(As[i].grad),
+        TL_TRY(bwd_impl(proj + i, rows, x[i], dY[i], nullptr, dX ? dX[i] : nullptr, const_cast<float *>(As[i].grad),
                         const_cast<float *>(Bs[i].grad), 0, c, false, st));
       }
     }
@@ -608,8 +627,8 @@ size_t templora_update_block_workspace_bytes(const templora_linear_t *proj, int3
   size_t need = 0, best = kStatusBytes;
   for (int mode = 0; mode < 2; ++mode) {
     t_path_override = mode;
-    update_impl(proj, nullptr, nullptr, n_proj, T, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0, 0, nullptr, nullptr,
-                0, true, &need, nullptr);
+    update_impl(proj, nullptr, nullptr, n_proj, T, T, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0, 0, nullptr,
+                nullptr, 0, true, &need, nullptr);
     if (need > best) best = need;
   }
   t_path_override = -1;
@@ -705,6 +724,17 @@ templora_status_t templora_update_block(const templora_linear_t *proj, const tem
                                         int32_t epochs, float lr, float beta1, float beta2, float eps,
                                         float weight_decay, int64_t *step_inout, void *ws, size_t ws_bytes,
                                         void *stream) {
+  return templora_update_block_batched(proj, A_state, B_state, n_proj, T, T, x, dY, y, dX, epochs, lr, beta1, beta2, eps,
+                                       weight_decay, step_inout, ws, ws_bytes, stream);
+}
+
+templora_status_t templora_update_block_batched(const templora_linear_t *proj, const templora_param_t *A_state,
+                                                const templora_param_t *B_state, int32_t n_proj, int32_t T,
+                                                int32_t batch_tokens, const void *const *x, const void *const *dY,
+                                                void *const *y, void *const *dX, int32_t epochs, float lr,
+                                                float beta1, float beta2, float eps, float weight_decay,
+                                                int64_t *step_inout, void *ws, size_t ws_bytes, void *stream) {
+  if (batch_tokens < 1) return TEMPLORA_ERR_INVALID_ARG;
   if (!proj || !A_state || !B_state || n_proj <= 0 || T <= 0 || !x || !dY || !y || epochs < 0 || !step_inout ||
       *step_inout < 0)
     return TEMPLORA_ERR_INVALID_ARG;
@@ -725,8 +755,8 @@ templora_status_t templora_update_block(const templora_linear_t *proj, const tem
     if (proj[i].A != wa || proj[i].B != wb) return TEMPLORA_ERR_INVALID_ARG;
   }
   TL_TRY(check_ws(ws, ws_bytes));
-  return update_impl(proj, A_state, B_state, n_proj, T, x, dY, y, dX, epochs, lr, beta1, beta2, eps, weight_decay,
-                     step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream));
+  return update_impl(proj, A_state, B_state, n_proj, T, batch_tokens, x, dY, y, dX, epochs, lr, beta1, beta2, eps,
+                     weight_decay, step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream));
 }
 
 const char *templora_status_string(templora_status_t st) {

@@ -332,3 +332,34 @@ def test_pins_catch_planted_mistakes():
         return fn
     for kind in ("dX_no_lora", "dB_no_s", "dA_uses_U", "dB_uses_V", "dA_mean"):
         assert not _pins_pass(f, bwd_variant(kind))
+
+
+def test_update_block_batches_are_sequential_updates_on_row_slices():
+    # chunk 10, batch 4, 2 epochs: 2 * ceil(10 / 4) = 6 optimizer steps (the cost table's count of
+    # training steps); by hand: one single-batch update per row slice, state carried along
+    projs = [_mk_proj(10, 6, 5, 2, 2.0), _mk_proj(10, 5, 7, 2, 2.0)]
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    st, step = orc.update_block(projs, 2, batch=4, **hp)
+    assert step == 6
+    cur = [dict(p) for p in projs]
+    k = 0
+    for _ in range(2):
+        for r0, r1 in ((0, 4), (4, 8), (8, 10)):
+            sl = [dict(c, x=c["x"][r0:r1], dY=c["dY"][r0:r1]) for c in cur]
+            out, k = orc.update_block(sl, 1, step0=k, **hp)
+            for c, o, full in zip(cur, out, st):
+                for key in ("A_master", "B_master", "mA", "vA", "mB", "vB"):
+                    c[key] = o[key]
+                last = o
+    assert k == 6
+    for c, full in zip(cur, st):
+        assert np.array_equal(c["A_master"], full["A_master"]) and np.array_equal(c["vB"], full["vB"])
+    # batch >= T is the unbatched update, bit for bit
+    a, _ = orc.update_block(projs, 2, **hp)
+    b, _ = orc.update_block(projs, 2, batch=10, **hp)
+    c, _ = orc.update_block(projs, 2, batch=64, **hp)
+    for u, v, w in zip(a, b, c):
+        assert np.array_equal(u["A_master"], v["A_master"]) and np.array_equal(u["y"], w["y"])
+    # rows of y come from the slice's own parameter version: the first slice of the last epoch
+    # was computed before the last two steps, so it differs from an unbatched pass with final weights
+    assert st[0]["y"].shape == (10, 5)

@@ -204,7 +204,7 @@ def test_adamw_many_tensors_one_call(b):
 
 
 # ------------------------------------------------------------------ update_block
-def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True):
+def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True, batch=None):
     hp = hp32(hp)
     hosts = [inputs.make_linear(seed, f"ub{i}", T, di, do, r, dtype=dtype) for i, (di, do) in enumerate(shapes)]
     devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
@@ -221,15 +221,21 @@ def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True
     ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(lins, T))
     args = b.UpdateBlockArgs(lins, As, Bs, [d["x"] for d in devs], [d["dY"] for d in devs], ys,
                              dXs if with_dX else None)
-    step = b.templora_update_block(args, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
-                                   0, ws)
+    if batch is None:
+        step = b.templora_update_block(args, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                       hp["weight_decay"], 0, ws)
+    else:
+        step = b.templora_update_block_batched(args, batch, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                               hp["weight_decay"], 0, ws)
     assert b.templora_read_device_status(ws)[0] == 0
-    assert step == epochs
+    n_steps = epochs * (1 if batch is None else -(-T // batch))
+    assert step == n_steps
     projs = [dict(x=f64(h["x"]), dY=f64(h["dY"]), W0=f64(h["W0"]), s=s, A_master=f64(h["A"]), B_master=f64(h["B"]))
              for h in hosts]
     ref, rstep = orc.update_block(projs, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
-                                  bf16_work=(dtype == "bf16"))
+                                  bf16_work=(dtype == "bf16"), batch=batch)
     assert rstep == step
+    epochs = n_steps   # below, "epochs" bounds the number of optimizer steps taken
     tol = TOL[dtype]
     for i, (q, st) in enumerate(zip(ref, states)):
         assert_close(f"y{i}", f64(ys[i]), q["y"], tol)
@@ -285,6 +291,19 @@ def test_update_block_more_projections_than_one_group(b):
 def test_update_block_generic_path(generic_path):
     _update_block_case(generic_path, "bf16", [(100, 60), (60, 100)], 33, 4, 2.0, 2,
                        dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01), 23)
+
+
+@pytest.mark.parametrize("T,batch", [(512, 256), (600, 256), (384, 128)])
+def test_update_block_batched_bf16(b, T, batch):
+    # chunk cut into batches: epochs * ceil(T / batch) optimizer steps, ragged last batch included
+    shapes = [(256, 384), (384, 256), (256, 256)]
+    _update_block_case(b, "bf16", shapes, T, 64, 2.0, 2, dict(lr=2e-4, beta1=0.9, beta2=0.999, eps=1e-8,
+                                                               weight_decay=0.0), 26, batch=batch)
+
+
+def test_update_block_batched_fp32(b):
+    _update_block_case(b, "f32", [(96, 80)], 70, 8, 2.0, 1, dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8,
+                                                                 weight_decay=0.01), 27, batch=32)
 
 
 def test_update_block_zero_epochs_is_a_no_op(b):

@@ -36,6 +36,22 @@ LLAMA2_70B_BLOCK = [  # grouped-query attention: k, v project to 1024
     ("gate", 8192, 28672), ("up", 8192, 28672), ("down", 28672, 8192),
 ]
 
+# other models the paper evaluates (Section "Experiments"): block shapes for the rank / chunk / batch sweeps
+LLAMA2_13B_BLOCK = [
+    ("q", 5120, 5120), ("k", 5120, 5120), ("v", 5120, 5120), ("o", 5120, 5120),
+    ("gate", 5120, 13824), ("up", 5120, 13824), ("down", 13824, 5120),
+]
+MISTRAL_7B_BLOCK = [  # grouped-query attention, 8 kv heads
+    ("q", 4096, 4096), ("k", 4096, 1024), ("v", 4096, 1024), ("o", 4096, 4096),
+    ("gate", 4096, 14336), ("up", 4096, 14336), ("down", 14336, 4096),
+]
+YI_6B_BLOCK = [  # grouped-query attention, 4 kv heads
+    ("q", 4096, 4096), ("k", 4096, 512), ("v", 4096, 512), ("o", 4096, 4096),
+    ("gate", 4096, 11008), ("up", 4096, 11008), ("down", 11008, 4096),
+]
+BLOCKS = {"llama2_7b": LLAMA2_7B_BLOCK, "llama2_13b": LLAMA2_13B_BLOCK, "llama2_70b": LLAMA2_70B_BLOCK,
+          "mistral_7b": MISTRAL_7B_BLOCK, "yi_6b": YI_6B_BLOCK}
+
 ADAMW = dict(lr=5e-5, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
 
 # The five workload configurations (index = configuration number).

@@ -149,3 +149,32 @@ def test_config3_decode_whole_block_in_one_call(b, n):
     for (W0, A, B), x, y in zip(keep, xs, ys):
         ref = orc.decode_fwd(f64(x), f64(W0), f64(A), f64(B), c["s"])
         assert_close(f"decode block n={n}", f64(y), ref, TOL["bf16"])
+
+
+# ------------------------------------------------------------------ the paper's other settings
+# chunk sizes 2048 and 4096 with smaller batches (several optimizer steps per epoch), rank 16..256,
+# 13B-shaped layers and grouped-query-attention shapes: full comparison against the oracle
+VARIANTS = [
+    ("llama2_13b", 2048, 1024, 16, 1),     # chunk 2048, batch 1024: 2 steps per epoch
+    ("mistral_7b", 1024, 1024, 256, 1),    # maximum rank, k/v project to 1024
+    ("yi_6b", 2048, 512, 64, 1),           # batch 512: 4 steps; k/v project to 512
+    ("llama2_7b", 1024, 256, 128, 2),      # batch 256, 2 epochs: 8 steps
+]
+
+
+@pytest.mark.parametrize("model,T,batch,r,epochs", VARIANTS)
+def test_variant_blocks_batched(b, model, T, batch, r, epochs):
+    from paper_2401_11504_b200 import runtime
+    hp = hp32(inputs.ADAMW)
+    blk = runtime.Block(b, 1, f"var/{model}", inputs.BLOCKS[model], T, r, 2.0, "bf16", "cuda")
+    projs0 = snapshot_block(blk)
+    ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(blk.lins, T))
+    step = b.templora_update_block_batched(blk.args, batch, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                           hp["weight_decay"], 0, ws)
+    assert b.templora_read_device_status(ws)[0] == 0
+    n_steps = epochs * -(-T // batch)
+    assert step == n_steps
+    ref, rstep = orc.update_block(projs0, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
+                                  bf16_work=True, batch=batch)
+    assert rstep == n_steps
+    compare_block(blk, projs0, ref, n_steps, hp["lr"])

@@ -184,6 +184,16 @@ const char *templora_status_string(templora_status_t st);
 templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *code, int32_t *where);
 
 /*
+ * Parallelized deployment (the paper's "Further Analysis": update the module in a second process or
+ * stream while generation continues, then swap it in).  Caps the number of SMs that the
+ * library's persistent kernels occupy when launched on `stream`, so that a chunk update on
+ * one stream and the decode-time forward on another run side by side instead of taking
+ * turns: e.g. 116 SMs for the update stream and 32 for the decode stream on a 148-SM B200.
+ * max_sms = 0 removes the cap.  Process-wide table keyed by the stream handle.
+ */
+templora_status_t templora_set_stream_sm_limit(void *stream, int32_t max_sms);
+
+/*
  * Kernel-path selection for testing: 0 = automatic (tensor-core path when the
  * shape allows, frozen-weight GEMMs on CTA pairs), 1 = always the generic kernel path,
  * 2 = tensor-core path with single-CTA tiles only.  Returns the previous value.

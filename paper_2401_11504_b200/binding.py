@@ -22,6 +22,7 @@ EXPORTS = [
     "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
     "templora_timing_enable", "templora_timing_read", "templora_decode_fwd_noalloc",
     "templora_decode_block_workspace_bytes", "templora_decode_block_fwd", "templora_update_block_batched",
+    "templora_set_stream_sm_limit",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH = range(7)
@@ -69,6 +70,8 @@ def _load():
     lib.templora_update_block_batched.restype = i32
     lib.templora_update_block_batched.argtypes = [LP, PP, PP, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                                   C.POINTER(vp), i32, f32, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_set_stream_sm_limit.restype = i32
+    lib.templora_set_stream_sm_limit.argtypes = [vp, i32]
     lib.templora_status_string.restype = C.c_char_p
     lib.templora_status_string.argtypes = [i32]
     lib.templora_read_device_status.restype = i32
@@ -275,3 +278,8 @@ class DecodeBlockArgs:
 def templora_decode_block_fwd(args, ws, stream=None):
     _check(lib.templora_decode_block_fwd(args.lins, args.n, args.n_tokens, args.x, args.y, _ptr(ws), ws.numel(),
                                          _stream(stream)), "templora_decode_block_fwd")
+
+
+def templora_set_stream_sm_limit(stream, max_sms):
+    """Cap the SMs the persistent kernels use on `stream` (0 = no cap)."""
+    _check(lib.templora_set_stream_sm_limit(_stream(stream), int(max_sms)), "templora_set_stream_sm_limit")

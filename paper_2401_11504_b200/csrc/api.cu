@@ -781,6 +781,12 @@ templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *c
   return TEMPLORA_OK;
 }
 
+templora_status_t templora_set_stream_sm_limit(void *stream, int32_t max_sms) {
+  if (max_sms < 0) return TEMPLORA_ERR_INVALID_ARG;
+  tc_set_stream_sm_limit(reinterpret_cast<cudaStream_t>(stream), max_sms);
+  return TEMPLORA_OK;
+}
+
 int32_t templora_set_kernel_path(int32_t mode) {
   return g_kernel_path.exchange((mode == 1 || mode == 2) ? mode : 0);
 }

@@ -148,6 +148,7 @@ constexpr int kTcMaxProblems = 16;
 templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st,
                                   int cta_pairs = 0);
 bool tc_available();
+void tc_set_stream_sm_limit(cudaStream_t st, int max_sms);
 
 // ---- workspace need of the decode-time forward alone (api.cu) -------------------
 size_t decode_workspace_need(const templora_linear_t *lin, int n);

@@ -22,6 +22,9 @@
 
 #include <cuda.h>
 
+#include <mutex>
+#include <unordered_map>
+
 namespace templora {
 namespace {
 
@@ -761,6 +764,17 @@ bool make_operand_map(CUtensorMap *m, const void *ptr, long long mn_extent, long
   return make_map(m, ptr, mn_extent, k_extent, ld, 64);
 }
 
+// Per-stream cap on the SMs the persistent kernels occupy (parallelized deployment: the chunk update
+// and the decode stream share the GPU).  0 / absent = no cap.
+std::mutex g_limit_mu;
+std::unordered_map<cudaStream_t, int> g_stream_limit;
+int stream_sm_limit(cudaStream_t st, int sm_count) {
+  std::lock_guard<std::mutex> lk(g_limit_mu);
+  auto it = g_stream_limit.find(st);
+  if (it == g_stream_limit.end() || it->second <= 0 || it->second > sm_count) return sm_count;
+  return it->second;
+}
+
 struct DeviceInfo {
   int sm_count = 0;
   int cc_major = 0;
@@ -788,7 +802,8 @@ templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream
     TL_CUDA_CHECK(cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes));
     di->attr_set[slot] = true;
   }
-  int grid = g.n_items < di->sm_count ? g.n_items : di->sm_count;
+  const int sms = stream_sm_limit(st, di->sm_count);
+  int grid = g.n_items < sms ? g.n_items : sms;
   {
     LaunchScope scope(BN == 256 ? kKindTcMain : (BN == 64 ? kKindTcSkinny : kKindTcDecode), st);
     TL_CUDA_CHECK(launch_pdl(tc_gemm_kernel<BN>, dim3(grid), dim3(kThreads), Cfg<BN>::kSmemBytes, st, g));
@@ -803,7 +818,8 @@ templora_status_t launch_pair(const DevGroup &g, DeviceInfo *di, cudaStream_t st
                                        pair::kSmemBytes));
     di->pair_attr_set = true;
   }
-  int pairs = di->sm_count / 2;
+  int pairs = stream_sm_limit(st, di->sm_count) / 2;
+  if (pairs < 1) pairs = 1;
   if (g.n_items < pairs) pairs = g.n_items;
   {
     LaunchScope scope(kKindTcMain, st);
@@ -814,6 +830,11 @@ templora_status_t launch_pair(const DevGroup &g, DeviceInfo *di, cudaStream_t st
 }
 
 }  // namespace
+
+void tc_set_stream_sm_limit(cudaStream_t st, int max_sms) {
+  std::lock_guard<std::mutex> lk(g_limit_mu);
+  if (max_sms <= 0) g_stream_limit.erase(st); else g_stream_limit[st] = max_sms;
+}
 
 bool tc_available() {
   DeviceInfo *di = device_info();

@@ -179,3 +179,63 @@ class ClockSampler:
         s = sorted(self.samples)
         return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
                 "samples": len(s)}
+
+
+# ------------------------------------------------------------------ parallelized deployment
+class ParallelDeployment:
+    """Chunk update and decode side by side on one GPU (the paper's parallelized deployment:
+    the module is updated elsewhere while generation goes on, then swapped in).
+
+    The update runs on its own stream and trains the block's working copies of A and B; decode runs
+    on another stream and reads separate *serving* copies, so it always sees a complete module.
+    publish() swaps the new module in at a decode-step boundary: on the decode stream, after the
+    update's completion event, the working copies are copied over the serving copies (10 MB for a
+    7B-shaped block).  Per-stream SM caps keep both persistent kernels resident at once.
+    Orchestration only: every product runs in the library's kernels.
+    """
+
+    def __init__(self, b, blk, n_tokens=1, update_sms=116, decode_sms=32, device="cuda"):
+        self.b, self.blk, self.n = b, blk, n_tokens
+        self.update_stream = torch.cuda.Stream(device=device)
+        self.decode_stream = torch.cuda.Stream(device=device)
+        b.templora_set_stream_sm_limit(self.update_stream, update_sms)
+        b.templora_set_stream_sm_limit(self.decode_stream, decode_sms)
+        self.serving = [(st["A"]["work"].clone(), st["B"]["work"].clone()) for st in blk.state]
+        self.lins = [b.linear_desc(W0, a, bb, blk.s) for W0, (a, bb) in zip(blk.W0, self.serving)]
+        td = blk.x[0].dtype
+        dt = "bf16" if td == torch.bfloat16 else "f32"
+        self.x = [inputs.make_tensor(0, "deploy", f"x{i}", (n_tokens, l.d_in), "normal", 1.0, dt, device)
+                  for i, l in enumerate(self.lins)]
+        self.y = [torch.empty((n_tokens, l.d_out), dtype=td, device=device) for l in self.lins]
+        self.dec_args = b.DecodeBlockArgs(self.lins, self.x, self.y)
+        self.ws_dec = b.alloc_workspace(b.templora_decode_block_workspace_bytes(self.lins), device)
+        self.ws_upd = b.alloc_workspace(b.templora_update_block_workspace_bytes(blk.lins, blk.T), device)
+        self.update_done = torch.cuda.Event()
+        self.published = torch.cuda.Event()
+        self.published.record(self.decode_stream)
+        self.step = 0
+
+    def start_update(self, epochs, hp, batch=None):
+        """Enqueue the chunk update on the update stream (returns at once)."""
+        self.update_stream.wait_event(self.published)   # the last publish has read the working copies
+        self.step = self.b.templora_update_block_batched(
+            self.blk.args, batch or self.blk.T, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+            hp["weight_decay"], self.step, self.ws_upd, stream=self.update_stream)
+        self.update_done.record(self.update_stream)
+
+    def decode_step(self):
+        """One decode-time forward of the whole block with the serving module."""
+        self.b.templora_decode_block_fwd(self.dec_args, self.ws_dec, stream=self.decode_stream)
+
+    def publish(self):
+        """Swap the updated module in between two decode steps."""
+        self.decode_stream.wait_event(self.update_done)
+        with torch.cuda.stream(self.decode_stream):
+            for st, (sa, sb) in zip(self.blk.state, self.serving):
+                sa.copy_(st["A"]["work"], non_blocking=True)
+                sb.copy_(st["B"]["work"], non_blocking=True)
+        self.published.record(self.decode_stream)
+
+    def close(self):
+        self.b.templora_set_stream_sm_limit(self.update_stream, 0)
+        self.b.templora_set_stream_sm_limit(self.decode_stream, 0)

@@ -291,7 +291,7 @@ def run_ours(args):
     # ---- decode-time LoRA GEMV bandwidth (second figure of the metric) -------
     decode = None
     if not args.no_decode:
-        decode = decode_bandwidth(b, torch, inputs, dev, peaks)
+        decode = decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=args.decode_blocks)
 
     # ---- parallelized deployment: the update on one stream, decode on another, SMs split ----
     parallel = None
@@ -339,26 +339,33 @@ def parallel_deployment(b, torch, runtime, blk, hp, update_sms=116, decode_sms=3
         upd = lambda: dep.start_update(1, hp)
         upd_alone_ms = timed(upd, dep.update_stream, n_updates)
         dec_alone_ms = timed(dep.decode_step, dep.decode_stream, 50)
-        # side by side: enqueue the updates, then decode until they are done
+        # side by side: enqueue the updates, then decode steps (each with its own event) well past their end;
+        # only the decode steps that finished while the updates were still running count as contended
         torch.cuda.synchronize()
-        e0, e1, d0, d1 = ev(), ev(), ev(), ev()
+        e0, e1 = ev(), ev()
+        n_dec = int(2.5 * n_updates * upd_alone_ms / max(dec_alone_ms, 1e-6)) + 8
+        marks = [ev() for _ in range(n_dec + 1)]
         e0.record(dep.update_stream)
         for _ in range(n_updates):
             upd()
         e1.record(dep.update_stream)
-        n_dec = int(1.2 * n_updates * upd_alone_ms / max(dec_alone_ms, 1e-6) * decode_sms / 148) + 8
-        d0.record(dep.decode_stream)
-        for _ in range(n_dec):
+        marks[0].record(dep.decode_stream)
+        for i in range(n_dec):
             dep.decode_step()
-        d1.record(dep.decode_stream)
+            marks[i + 1].record(dep.decode_stream)
         torch.cuda.synchronize()
+        upd_end = marks[0].elapsed_time(e1)                      # update end on the decode stream's clock
+        ends = [marks[0].elapsed_time(m) for m in marks[1:]]
+        contended = [i for i, t in enumerate(ends) if t <= upd_end]
+        dec_side_us = (ends[contended[-1]] / (contended[-1] + 1) * 1e3) if contended else None
         dep.publish()
         torch.cuda.synchronize()
         return {"update_sms": update_sms, "decode_sms": decode_sms,
                 "update_ms_alone_capped": upd_alone_ms, "decode_step_us_alone_capped": dec_alone_ms * 1e3,
                 "update_ms_side_by_side": e0.elapsed_time(e1) / n_updates,
-                "decode_step_us_side_by_side": d0.elapsed_time(d1) / n_dec * 1e3, "decode_steps": n_dec,
-                "note": "both streams keep their SM caps in the 'alone' figures; whether the two windows overlapped fully depends on n_dec"}
+                "decode_step_us_side_by_side": dec_side_us, "decode_steps_during_updates": len(contended),
+                "what": "7B block: chunk updates (T=1024) back to back on one stream, single-token decode steps of the "
+                        "same block on another; 'alone' figures keep the SM caps"}
     finally:
         dep.close()
 
@@ -444,6 +451,7 @@ def main():
     ap.add_argument("--rank", type=int, default=64)
     ap.add_argument("--epochs", type=int, default=1)
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--decode-blocks", type=int, default=32, help="distinct blocks the decode measurement rotates over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parallel", action="store_true", help="skip the parallelized-deployment measurement")
     args = ap.parse_args()

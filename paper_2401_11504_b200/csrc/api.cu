@@ -283,6 +283,8 @@ struct FinishBatch {
 constexpr int kFinO = 64;
 constexpr int kFinTy = 4;   // 256 threads per block: the whole grid (d_out / 64 blocks) is resident at once
 
+// TOK = tokens per thread: 1 when n <= kFinTy (every token has its own lane), else 4.
+template <int TOK>
 __global__ void __launch_bounds__(kFinO * kFinTy, 6) decode_finish_kernel(const __grid_constant__ FinishBatch fb) {
   extern __shared__ __align__(16) uint8_t fin_smem[];
   pdl_prologue();
@@ -304,30 +306,65 @@ __global__ void __launch_bounds__(kFinO * kFinTy, 6) decode_finish_kernel(const 
     if (o0 + row < d_out) w = *reinterpret_cast<const uint4 *>(f.B + (long long)(o0 + row) * r + ch * 8);
     *reinterpret_cast<uint4 *>(b_sm + row * pitch + ch * 8) = w;
   }
-  for (int e = tid; e < n * r; e += nthreads) {
-    float a = 0.f;
-    for (int k = 0; k < f.spu; ++k) a += f.Pu[(long long)k * n * r + e];
-    u_sm[e] = f.s * a;
+  for (int e0 = tid; e0 < n * r; e0 += 4 * nthreads) {   // four elements per thread per pass, loads batched
+    float a[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k = 0; k < f.spu; ++k) {
+      const float *src = f.Pu + (long long)k * n * r;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int e = e0 + q * nthreads;
+        if (e < n * r) a[q] += __ldg(src + e);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int e = e0 + q * nthreads;
+      if (e < n * r) u_sm[e] = f.s * a[q];
+    }
   }
   __syncthreads();
   const int o = o0 + threadIdx.x;
   if (o >= d_out) return;
   const __nv_bfloat16 *brow = b_sm + threadIdx.x * pitch;
-  for (int i = threadIdx.y; i < n; i += blockDim.y) {
-    float acc = 0.f;
-    for (int k = 0; k < f.sp; ++k) acc += f.P[((long long)k * n + i) * d_out + o];
-    const float *urow = u_sm + i * r;
-    for (int j0 = 0; j0 < r; j0 += 8) {
-      const uint4 w = *reinterpret_cast<const uint4 *>(brow + j0);
-      const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&w);
-      const float4 u0 = *reinterpret_cast<const float4 *>(urow + j0);       // same address across the warp
-      const float4 u1 = *reinterpret_cast<const float4 *>(urow + j0 + 4);
-      const float2 b0 = __bfloat1622float2(h[0]), b1 = __bfloat1622float2(h[1]);
-      const float2 b2 = __bfloat1622float2(h[2]), b3 = __bfloat1622float2(h[3]);
-      acc = fmaf(u0.x, b0.x, acc); acc = fmaf(u0.y, b0.y, acc); acc = fmaf(u0.z, b1.x, acc); acc = fmaf(u0.w, b1.y, acc);
-      acc = fmaf(u1.x, b2.x, acc); acc = fmaf(u1.y, b2.y, acc); acc = fmaf(u1.z, b3.x, acc); acc = fmaf(u1.w, b3.y, acc);
+  // tokens threadIdx.y, +kFinTy, ... (at most four): all their slab loads are issued before any is used,
+  // so the slabs (usually evicted to DRAM by the W0 stream) cost one memory latency per slab, not per token
+  float acc[TOK];
+#pragma unroll
+  for (int q = 0; q < TOK; ++q) acc[q] = 0.f;
+  for (int k = 0; k < f.sp; ++k) {
+    const float *src = f.P + (long long)k * n * d_out + o;
+    float t[TOK];
+#pragma unroll
+    for (int q = 0; q < TOK; ++q) {
+      const int i = threadIdx.y + q * kFinTy;
+      t[q] = (i < n) ? __ldg(src + (long long)i * d_out) : 0.f;
     }
-    f.y[(long long)i * d_out + o] = __float2bfloat16_rn(acc);
+#pragma unroll
+    for (int q = 0; q < TOK; ++q) acc[q] += t[q];
+  }
+  for (int j0 = 0; j0 < r; j0 += 8) {
+    const uint4 w = *reinterpret_cast<const uint4 *>(brow + j0);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&w);
+    const float2 b0 = __bfloat1622float2(h[0]), b1 = __bfloat1622float2(h[1]);
+    const float2 b2 = __bfloat1622float2(h[2]), b3 = __bfloat1622float2(h[3]);
+#pragma unroll
+    for (int q = 0; q < TOK; ++q) {
+      const int i = threadIdx.y + q * kFinTy;
+      if (i < n) {
+        const float *urow = u_sm + i * r + j0;
+        const float4 u0 = *reinterpret_cast<const float4 *>(urow);       // same address across the warp
+        const float4 u1 = *reinterpret_cast<const float4 *>(urow + 4);
+        float a = acc[q];
+        a = fmaf(u0.x, b0.x, a); a = fmaf(u0.y, b0.y, a); a = fmaf(u0.z, b1.x, a); a = fmaf(u0.w, b1.y, a);
+        a = fmaf(u1.x, b2.x, a); a = fmaf(u1.y, b2.y, a); a = fmaf(u1.z, b3.x, a); a = fmaf(u1.w, b3.y, a);
+        acc[q] = a;
+      }
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < TOK; ++q) {
+    const int i = threadIdx.y + q * kFinTy;
+    if (i < n) f.y[(long long)i * d_out + o] = __float2bfloat16_rn(acc[q]);
   }
 }
 
@@ -393,11 +430,16 @@ templora_status_t decode_group_tc(const templora_linear_t *proj, int np, int n, 
     TL_CUDA_CHECK(cudaGetDevice(&dev_id));
     bool &attr_done = attr_done_dev[dev_id & 63];
     if (!attr_done) {
-      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
-      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50));
+      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel<1>, cudaFuncAttributePreferredSharedMemoryCarveout, 50));
+      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+      TL_CUDA_CHECK(cudaFuncSetAttribute(decode_finish_kernel<4>, cudaFuncAttributePreferredSharedMemoryCarveout, 50));
       attr_done = true;
     }
-    TL_CUDA_CHECK(launch_pdl(decode_finish_kernel, dim3(blocks), dim3(kFinO, kFinTy), smem, st, fb));
+    if (n <= kFinTy)
+      TL_CUDA_CHECK(launch_pdl(decode_finish_kernel<1>, dim3(blocks), dim3(kFinO, kFinTy), smem, st, fb));
+    else
+      TL_CUDA_CHECK(launch_pdl(decode_finish_kernel<4>, dim3(blocks), dim3(kFinO, kFinTy), smem, st, fb));
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;

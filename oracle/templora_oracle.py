@@ -19,6 +19,13 @@ n = 2 epochs, bfloat16 training):
     dA = s V^T x                       [r, d_in]
     (W0 is frozen: the method never alters the base model, so no dW0 exists.)
 
+With LoRA dropout (paper's Setup: dropout = 0.05; in LoRA the dropout sits on the input of
+the low-rank branch) the branch reads xd = x * keep / (1 - p) instead of x:
+    U = xd A^T ;  dA = s V^T xd ;  dX = dY W0 + s (V A) * keep / (1 - p) ;  y, V, dB as above.
+keep[t,k] in {0,1} comes from the counter-based generator Philox4x32-10 (Salmon, Moraes, Dror,
+Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11), written out below from its
+published definition.
+
 Every function is the definition written out with numpy matmuls on float64
 arrays, in the order above; nothing is blocked, fused or reordered.
 
@@ -45,10 +52,12 @@ def _f64(a):
 # --------------------------------------------------------------------------
 # forward:  y = x W0^T + s (x A^T) B^T            (Temp-Lora module forward)
 # --------------------------------------------------------------------------
-def linear_fwd(x, W0, A, B, s):
-    """x [T,d_in], W0 [d_out,d_in], A [r,d_in], B [d_out,r] -> (y [T,d_out], U [T,r])."""
+def linear_fwd(x, W0, A, B, s, keep=None, p=0.0):
+    """x [T,d_in], W0 [d_out,d_in], A [r,d_in], B [d_out,r] -> (y [T,d_out], U [T,r]).
+    keep [T,d_in] of 0/1 and p: LoRA dropout on the input of the low-rank branch."""
     x, W0, A, B = _f64(x), _f64(W0), _f64(A), _f64(B)
-    U = x @ A.T
+    xd = x if keep is None else x * _f64(keep) / (1.0 - F64(p))
+    U = xd @ A.T
     y = x @ W0.T + F64(s) * (U @ B.T)
     return y, U
 
@@ -56,16 +65,58 @@ def linear_fwd(x, W0, A, B, s):
 # --------------------------------------------------------------------------
 # backward with W0 frozen (no dW0: the base model is never altered)
 # --------------------------------------------------------------------------
-def linear_bwd(x, dY, W0, A, B, s):
+def linear_bwd(x, dY, W0, A, B, s, keep=None, p=0.0):
     """-> (dX [T,d_in], dA [r,d_in], dB [d_out,r]); gradients are plain sums over tokens."""
     x, dY, W0, A, B = _f64(x), _f64(dY), _f64(W0), _f64(A), _f64(B)
     s = F64(s)
-    U = x @ A.T
+    scale = 1.0 if keep is None else _f64(keep) / (1.0 - F64(p))   # d xd / d x, elementwise
+    xd = x * scale
+    U = xd @ A.T
     V = dY @ B
-    dX = dY @ W0 + s * (V @ A)
+    dX = dY @ W0 + s * (V @ A) * scale
     dB = s * (dY.T @ U)
-    dA = s * (V.T @ x)
+    dA = s * (V.T @ xd)
     return dX, dA, dB
+
+
+# --------------------------------------------------------------------------
+# Philox4x32-10 and the dropout mask drawn from it
+# --------------------------------------------------------------------------
+_PHILOX_M0, _PHILOX_M1 = np.uint64(0xD2511F53), np.uint64(0xCD9E8D57)
+_PHILOX_W0, _PHILOX_W1 = np.uint64(0x9E3779B9), np.uint64(0xBB67AE85)
+_MASK32 = np.uint64(0xFFFFFFFF)
+
+
+def philox4x32_10(counter, key):
+    """counter: uint32 array [..., 4], key: (k0, k1).  Ten rounds of
+        (c0, c1, c2, c3) <- (hi(M1*c2) ^ c1 ^ k0,  lo(M1*c2),  hi(M0*c0) ^ c3 ^ k1,  lo(M0*c0))
+    with the key bumped by the Weyl constants after every round.  Returns uint32 [..., 4]."""
+    c = np.asarray(counter, dtype=np.uint64)
+    c0, c1, c2, c3 = c[..., 0], c[..., 1], c[..., 2], c[..., 3]
+    k0, k1 = np.uint64(int(key[0]) & 0xFFFFFFFF), np.uint64(int(key[1]) & 0xFFFFFFFF)
+    for _ in range(10):
+        p0, p1 = _PHILOX_M0 * c0, _PHILOX_M1 * c2          # 32 x 32 -> 64 bit products
+        c0, c1, c2, c3 = ((p1 >> np.uint64(32)) ^ c1 ^ k0, p1 & _MASK32,
+                          (p0 >> np.uint64(32)) ^ c3 ^ k1, p0 & _MASK32)
+        k0, k1 = (k0 + _PHILOX_W0) & _MASK32, (k1 + _PHILOX_W1) & _MASK32
+    return np.stack([c0, c1, c2, c3], axis=-1).astype(np.uint32)
+
+
+def dropout_threshold(p):
+    """An element is dropped iff its 32-bit draw is below floor(p * 2^32)."""
+    return int(np.floor(float(p) * 4294967296.0))
+
+
+def dropout_keep(seed, offset, T, d_in, p):
+    """keep [T, d_in] of 0/1.  Element e = t*d_in + k takes word e % 4 of
+    Philox4x32-10(counter = (lo(e/4), hi(e/4), lo(offset), hi(offset)), key = (lo(seed), hi(seed)))."""
+    n = int(T) * int(d_in)
+    q = np.arange((n + 3) // 4, dtype=np.uint64)
+    ctr = np.empty((q.size, 4), dtype=np.uint64)
+    ctr[:, 0], ctr[:, 1] = q & _MASK32, q >> np.uint64(32)
+    ctr[:, 2], ctr[:, 3] = np.uint64(int(offset) & 0xFFFFFFFF), np.uint64((int(offset) >> 32) & 0xFFFFFFFF)
+    draws = philox4x32_10(ctr, (int(seed) & 0xFFFFFFFF, (int(seed) >> 32) & 0xFFFFFFFF)).reshape(-1)[:n]
+    return (draws >= np.uint32(min(dropout_threshold(p), 0xFFFFFFFF))).astype(np.uint8).reshape(int(T), int(d_in))
 
 
 # --------------------------------------------------------------------------
@@ -116,7 +167,8 @@ def round_bf16(a):
 # the whole update of one block of projections: n epochs over the chunk,
 # one optimizer step per epoch (batch = chunk)
 # --------------------------------------------------------------------------
-def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf16_work=False, batch=None):
+def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf16_work=False, batch=None,
+                 dropout_p=0.0):
     """projs: list of dicts with keys x, dY, W0, s, A_master, B_master and optionally
     mA, vA, mB, vB (default 0).  For each epoch: forward and backward of every
     projection with the current working A, B; then step += 1 and AdamW on every
@@ -125,7 +177,9 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
     training under ZeRO-2 implies).  With batch < T every epoch walks the chunk in
     row slices of `batch` tokens and takes one optimizer step per slice (the cost
     table's "training steps" = epochs * chunk / batch); y and dX are then filled
-    slice by slice and dA, dB are the last slice's.
+    slice by slice and dA, dB are the last slice's.  With dropout_p > 0 every optimizer step
+    draws a fresh mask for its row slice: projection i uses seed projs[i]["dropout_seed"]
+    and offset projs[i].get("dropout_offset", 0) + (number of steps taken before this one).
 
     Returns (state, step): state[i] has A_master, B_master, mA, vA, mB, vB and the
     last epoch's y, dX, dA, dB.
@@ -150,8 +204,12 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
                 A = round_bf16(q["A_master"]) if bf16_work else q["A_master"]
                 B = round_bf16(q["B_master"]) if bf16_work else q["B_master"]
                 xb, dYb = _f64(p["x"])[rows], _f64(p["dY"])[rows]
-                q["y"][rows], _ = linear_fwd(xb, p["W0"], A, B, p["s"])
-                q["dX"][rows], q["dA"], q["dB"] = linear_bwd(xb, dYb, p["W0"], A, B, p["s"])
+                keep = None
+                if dropout_p > 0:
+                    keep = dropout_keep(p["dropout_seed"], p.get("dropout_offset", 0) + step, xb.shape[0],
+                                        xb.shape[1], dropout_p)
+                q["y"][rows], _ = linear_fwd(xb, p["W0"], A, B, p["s"], keep, dropout_p)
+                q["dX"][rows], q["dA"], q["dB"] = linear_bwd(xb, dYb, p["W0"], A, B, p["s"], keep, dropout_p)
             step += 1
             for q in st:
                 q["A_master"], q["mA"], q["vA"] = adamw_step(q["A_master"], q["dA"], q["mA"], q["vA"],

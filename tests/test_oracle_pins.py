@@ -363,3 +363,83 @@ def test_update_block_batches_are_sequential_updates_on_row_slices():
     # rows of y come from the slice's own parameter version: the first slice of the last epoch
     # was computed before the last two steps, so it differs from an unbatched pass with final weights
     assert st[0]["y"].shape == (10, 5)
+
+
+# ------------------------------------------------------------------- dropout
+def test_philox4x32_10_known_answers():
+    # known-answer vectors published with the generator (Random123 distribution, kat_vectors)
+    kat = [
+        ((0, 0, 0, 0), (0, 0), (0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8)),
+        ((0xffffffff,) * 4, (0xffffffff, 0xffffffff), (0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd)),
+        ((0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344), (0xa4093822, 0x299f31d0),
+         (0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1)),
+    ]
+    for ctr, key, want in kat:
+        got = orc.philox4x32_10(np.array([ctr], dtype=np.uint32), key)[0]
+        assert tuple(int(v) for v in got) == want
+
+
+def test_dropout_keep_statistics_and_determinism():
+    k1 = orc.dropout_keep(1234, 7, 300, 512, 0.05)
+    assert k1.shape == (300, 512) and set(np.unique(k1)) <= {0, 1}
+    assert abs(k1.mean() - 0.95) < 0.005                      # 153600 draws: sigma = 5.6e-4
+    assert np.array_equal(k1, orc.dropout_keep(1234, 7, 300, 512, 0.05))
+    assert not np.array_equal(k1, orc.dropout_keep(1234, 8, 300, 512, 0.05))     # next step, new mask
+    assert not np.array_equal(k1, orc.dropout_keep(1235, 7, 300, 512, 0.05))
+    assert orc.dropout_keep(1, 0, 8, 8, 0.0).all()
+    # a larger p only drops more: same draws, higher threshold
+    k5 = orc.dropout_keep(1234, 7, 300, 512, 0.5)
+    assert abs(k5.mean() - 0.5) < 0.01 and not (k5 & ~k1).any()
+    # a row slice of a longer chunk is NOT the same mask (the element index depends on the slice shape)
+    assert orc.dropout_keep(9, 0, 4, 16, 0.3).shape == (4, 16)
+
+
+def test_dropout_forward_backward_against_loops_and_differences():
+    T, d_in, d_out, r, s, p = 5, 8, 6, 3, 2.0, 0.25
+    x, W0, A, B, dY = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r), rnd(T, d_out)
+    keep = orc.dropout_keep(77, 3, T, d_in, p)
+    assert 0 < keep.sum() < keep.size
+    y, U = orc.linear_fwd(x, W0, A, B, s, keep, p)
+    # scalar loops
+    for t in range(T):
+        u = [sum(x[t][k] * keep[t][k] / (1 - p) * A[j][k] for k in range(d_in)) for j in range(r)]
+        for o in range(d_out):
+            want = sum(x[t][k] * W0[o][k] for k in range(d_in)) + s * sum(u[j] * B[o][j] for j in range(r))
+            assert abs(y[t][o] - want) < 1e-12
+    # the loss sum(dY*y) stays linear in each of x, A, B with the mask held fixed: exact differences
+    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, s, keep, p)
+    loss = lambda xx, AA, BB: float((dY * orc.linear_fwd(xx, W0, AA, BB, s, keep, p)[0]).sum())
+    h = 0.5
+    for arr, grad, which in ((x, dX, 0), (A, dA, 1), (B, dB, 2)):
+        fd = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            plus, minus = arr.copy(), arr.copy()
+            plus[idx] += h; minus[idx] -= h
+            args_p, args_m = [x, A, B], [x, A, B]
+            args_p[which], args_m[which] = plus, minus
+            fd[idx] = (loss(*args_p) - loss(*args_m)) / (2 * h)
+        assert np.abs(grad - fd).max() <= 1e-9 * max(1.0, np.abs(fd).max())
+    # p = 0 / no mask is the plain projection, bit for bit; an all-ones mask with p = 0 too
+    y0, _ = orc.linear_fwd(x, W0, A, B, s)
+    y1, _ = orc.linear_fwd(x, W0, A, B, s, np.ones_like(keep), 0.0)
+    assert np.array_equal(y0, y1)
+    # dropped inputs get no gradient through the LoRA branch
+    base = dY @ W0
+    assert np.allclose((dX - base)[keep == 0], 0.0)
+
+
+def test_update_block_with_dropout_draws_a_mask_per_step():
+    projs = [dict(_mk_proj(8, 8, 6, 2, 2.0), dropout_seed=5), dict(_mk_proj(8, 6, 8, 2, 2.0), dropout_seed=6)]
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    st, step = orc.update_block(projs, 2, dropout_p=0.5, batch=4, **hp)
+    assert step == 4
+    # by hand for the first step of projection 0: rows 0..3, offset 0 + 0 steps taken
+    keep = orc.dropout_keep(5, 0, 4, 8, 0.5)
+    p = projs[0]
+    _, dA, dB = orc.linear_bwd(p["x"][:4], p["dY"][:4], p["W0"], p["A_master"], p["B_master"], 2.0, keep, 0.5)
+    A1, _, _ = orc.adamw_step(p["A_master"], dA, 0 * dA, 0 * dA, t=1, **hp)
+    one, _ = orc.update_block([dict(p, x=p["x"][:4], dY=p["dY"][:4])], 1, dropout_p=0.5, **hp)
+    assert np.array_equal(one[0]["A_master"], A1)
+    # and dropout changes the result
+    plain, _ = orc.update_block(projs, 2, batch=4, **hp)
+    assert np.abs(plain[0]["A_master"] - st[0]["A_master"]).max() > 0

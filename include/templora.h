@@ -63,6 +63,18 @@ typedef struct {
   const void *W0;     /* [d_out, d_in]  frozen, read only                           */
   const void *A;      /* [r, d_in]      working copy in `dtype`                     */
   const void *B;      /* [d_out, r]     working copy in `dtype`                     */
+  /* LoRA dropout on the input of the low-rank branch during the update (paper's Setup:
+   * dropout = 0.05).  0 disables it.  The keep mask of an [T, d_in] input is drawn from
+   * Philox4x32-10: element e = t*d_in + k takes word e % 4 of the block with counter
+   * (lo(e/4), hi(e/4), lo(offset), hi(offset)) and key (lo(seed), hi(seed)), and is dropped
+   * iff that word < floor(p * 2^32).  templora_linear_fwd and templora_linear_bwd use
+   * offset = dropout_offset (pass the same value to both); templora_update_block adds the
+   * number of optimizer steps already taken, so every step draws a new mask.  The
+   * decode-time forward never drops.  */
+  float dropout_p;
+  int32_t reserved;
+  uint64_t dropout_seed;
+  uint64_t dropout_offset;
 } templora_linear_t;
 
 /* Optimizer state of one tensor (an A or a B); all buffers caller-owned, n elements. */
@@ -87,6 +99,7 @@ size_t templora_update_block_workspace_bytes(const templora_linear_t *proj, int3
  * Forward of the LoRA-augmented projection over a chunk of T tokens
  * (module forward inside "Train Theta_k", Algorithm 1; LoRA of the Section "Temp-Lora"):
  *     U = x A^T ;  y = x W0^T + s U B^T
+ * (with dropout_p > 0:  U = xd A^T,  xd = x * keep / (1 - p))
  * x [T,d_in] in, y [T,d_out] out.  U_save: optional fp32 [T,r] that receives U
  * (unscaled) for reuse by templora_linear_bwd; NULL to skip.
  */
@@ -97,6 +110,7 @@ templora_status_t templora_linear_fwd(const templora_linear_t *lin, int32_t T, c
  * Backward of the same projection with W0 frozen (the method never alters the base
  * model, so there is no dW0):
  *     V = dY B ;  dX = dY W0 + s V A ;  dB = s dY^T U ;  dA = s V^T x
+ * (with dropout_p > 0:  dX = dY W0 + s (V A) * keep / (1 - p),  dA = s V^T xd)
  * U_saved: fp32 [T,r] from the forward, or NULL to recompute U = x A^T.
  * dX [T,d_in] may be NULL (skipped).  dA [r,d_in], dB [d_out,r] are fp32 and are
  * plain sums over the T tokens (no 1/T); accumulate != 0 adds to their contents.

@@ -54,6 +54,7 @@ templora_status_t check_linear(const templora_linear_t *lin) {
   if (lin->dtype != TEMPLORA_F32 && lin->dtype != TEMPLORA_BF16) return TEMPLORA_ERR_UNSUPPORTED;
   if (lin->r > 256) return TEMPLORA_ERR_UNSUPPORTED;
   if (!(lin->s == lin->s)) return TEMPLORA_ERR_INVALID_ARG;
+  if (!(lin->dropout_p >= 0.f && lin->dropout_p < 1.f)) return TEMPLORA_ERR_INVALID_ARG;
   return TEMPLORA_OK;
 }
 templora_status_t check_linear_ptrs(const templora_linear_t *lin) {
@@ -137,6 +138,37 @@ TcProblem prob_dA(const templora_linear_t *l, int T, const void *x, const void *
 int splits_skinny(int T, int r, int K, int group) { return pick_splits(cdiv(T, 128) * cdiv(r, 64), cdiv(K, 64), group); }
 int splits_grad(int d, int r, int T, int group) { return pick_splits(cdiv(d, 128) * cdiv(r, 64), cdiv(T, 64), group); }
 
+// ---------------------------------------------------------------- dropout scratch
+struct DropBufs {
+  void *xd = nullptr;        // x * keep / (1 - p), storage type of x
+  uint8_t *mask = nullptr;   // keep bits
+  long long pitch = 0;
+};
+DropBufs take_drop(const templora_linear_t *l, int T, WsAlloc &ws) {
+  DropBufs d;
+  if (l->dropout_p > 0.f) {
+    const size_t esize = l->dtype == TEMPLORA_BF16 ? 2 : 4;
+    d.xd = ws.take<uint8_t>((size_t)T * l->d_in * esize);
+    d.pitch = dropout_mask_pitch(l->d_in);
+    d.mask = ws.take<uint8_t>((size_t)T * d.pitch);
+  }
+  return d;
+}
+DropoutJob drop_job(const templora_linear_t *l, int T, const void *x, const DropBufs &d, uint64_t step_offset) {
+  return DropoutJob{x, d.xd, d.mask, T, l->d_in, d.pitch, l->dtype, l->dropout_p, l->dropout_seed,
+                    l->dropout_offset + step_offset};
+}
+// dX += keep * (s / (1 - p)) * (V A): one pass over dX on 128 x 256 tiles with a single k-block
+TcProblem prob_dX_dropout_term(const templora_linear_t *l, int T, const void *Vs, void *dX, const DropBufs &d) {
+  TcProblem p{};
+  p.M = T; p.N = l->d_in; p.K = l->r;
+  p.A = Vs; p.lda = l->r; p.a_mn = 0;
+  p.B = l->A; p.ldb = l->d_in; p.b_mn = 1;
+  p.splits = 1; p.out = dX; p.out_f32 = 0; p.out_s0 = l->d_in; p.out_s1 = 1;
+  p.epi_mask = d.mask; p.epi_mask_pitch = d.pitch; p.epi_scale = (float)(1.0 / (1.0 - (double)l->dropout_p));
+  return p;
+}
+
 // ---------------------------------------------------------------- forward
 templora_status_t fwd_impl(const templora_linear_t *l, int T, const void *x, void *y, float *U_save, WsAlloc &ws,
                            bool dry, cudaStream_t st) {
@@ -145,9 +177,14 @@ templora_status_t fwd_impl(const templora_linear_t *l, int T, const void *x, voi
     const int su = splits_skinny(T, l->r, l->d_in, 1);
     float *Upart = ws.take<float>((size_t)su * Tr);
     __nv_bfloat16 *Us = ws.take<__nv_bfloat16>((size_t)Tr);
+    const DropBufs drop = take_drop(l, T, ws);
     if (dry) return TEMPLORA_OK;
     if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
-    TcProblem pu = prob_U(l, T, x, Upart, su);
+    if (drop.xd) {
+      DropoutJob dj = drop_job(l, T, x, drop, 0);
+      TL_TRY(dropout_apply_batch(&dj, 1, st));
+    }
+    TcProblem pu = prob_U(l, T, drop.xd ? drop.xd : x, Upart, su);
     TL_TRY(tc_gemm_grouped(&pu, 1, 64, ws.status(), st));
     ReduceJob rj{Upart, su, Tr, Tr, l->s, 1.f, U_save, 0, Us};
     TL_TRY(reduce_partials_batch(&rj, 1, st));
@@ -155,12 +192,17 @@ templora_status_t fwd_impl(const templora_linear_t *l, int T, const void *x, voi
     return tc_gemm_grouped(&py, 1, 256, ws.status(), st, use_pairs());
   }
   float *U = U_save ? U_save : ws.take<float>((size_t)Tr);
+  const DropBufs drop = take_drop(l, T, ws);
   if (dry) return TEMPLORA_OK;
   if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
   const int dt = l->dtype;
+  if (drop.xd) {
+    DropoutJob dj = drop_job(l, T, x, drop, 0);
+    TL_TRY(dropout_apply_batch(&dj, 1, st));
+  }
   SimtGemm g{};
   g.M = T; g.N = l->r; g.K1 = l->d_in; g.K2 = 0;
-  g.A1 = op(x, dt, l->d_in, 1); g.B1 = op(l->A, dt, 1, l->d_in);
+  g.A1 = op(drop.xd ? drop.xd : x, dt, l->d_in, 1); g.B1 = op(l->A, dt, 1, l->d_in);
   g.alpha1 = 1.f; g.alpha2 = 0.f; g.D = U; g.d_dt = TEMPLORA_F32; g.ds0 = l->r; g.ds1 = 1;
   TL_TRY(simt_gemm(g, st));
   SimtGemm h{};
@@ -186,13 +228,19 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
     const bool direct_b = (sb == 1 && !accumulate), direct_a = (sa == 1 && !accumulate);
     float *dBpart = direct_b ? dB : ws.take<float>((size_t)sb * l->d_out * l->r);
     float *dApart = direct_a ? dA : ws.take<float>((size_t)sa * l->d_in * l->r);
+    const DropBufs drop = take_drop(l, T, ws);
     if (dry) return TEMPLORA_OK;
     if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+    if (drop.xd) {   // the same mask as the forward's: same seed, same offset, same shape
+      DropoutJob dj = drop_job(l, T, x, drop, 0);
+      TL_TRY(dropout_apply_batch(&dj, 1, st));
+    }
+    const void *xb = drop.xd ? drop.xd : x;   // what the low-rank branch read
 
     TcProblem skinny[2];
     int ns = 0;
     skinny[ns++] = prob_V(l, T, dY, Vpart, sv);
-    if (!U_saved) skinny[ns++] = prob_U(l, T, x, Upart, su);
+    if (!U_saved) skinny[ns++] = prob_U(l, T, xb, Upart, su);
     TL_TRY(tc_gemm_grouped(skinny, ns, 64, ws.status(), st));
     ReduceJob jobs[2] = {
         ReduceJob{Vpart, sv, Tr, Tr, l->s, 1.f, nullptr, 0, Vs},
@@ -201,9 +249,14 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
     TL_TRY(reduce_partials_batch(jobs, 2, st));
     if (dX) {
       TcProblem px = prob_dX(l, T, dY, Vs, dX);
+      if (drop.xd) px.Kext = 0;   // the rank-r term is masked per element: added by a second pass
       TL_TRY(tc_gemm_grouped(&px, 1, 256, ws.status(), st, use_pairs()));
+      if (drop.xd) {
+        TcProblem pt = prob_dX_dropout_term(l, T, Vs, dX, drop);
+        TL_TRY(tc_gemm_grouped(&pt, 1, 256, ws.status(), st, 0));
+      }
     }
-    TcProblem grads[2] = {prob_dB(l, T, dY, Us, dBpart, sb), prob_dA(l, T, x, Vs, dApart, sa)};
+    TcProblem grads[2] = {prob_dB(l, T, dY, Us, dBpart, sb), prob_dA(l, T, xb, Vs, dApart, sa)};
     TL_TRY(tc_gemm_grouped(grads, 2, 64, ws.status(), st));
     ReduceJob rj[2];
     int nr = 0;
@@ -215,14 +268,20 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
   }
   float *Ubuf = U_saved ? nullptr : ws.take<float>((size_t)Tr);
   float *V = ws.take<float>((size_t)Tr);
+  const DropBufs drop = take_drop(l, T, ws);
   if (dry) return TEMPLORA_OK;
   if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
   const int dt = l->dtype;
+  if (drop.xd) {
+    DropoutJob dj = drop_job(l, T, x, drop, 0);
+    TL_TRY(dropout_apply_batch(&dj, 1, st));
+  }
+  const void *xb = drop.xd ? drop.xd : x;
   const float *U = U_saved;
   if (!U) {
     SimtGemm g{};
     g.M = T; g.N = l->r; g.K1 = l->d_in;
-    g.A1 = op(x, dt, l->d_in, 1); g.B1 = op(l->A, dt, 1, l->d_in);
+    g.A1 = op(xb, dt, l->d_in, 1); g.B1 = op(l->A, dt, 1, l->d_in);
     g.alpha1 = 1.f; g.D = Ubuf; g.d_dt = TEMPLORA_F32; g.ds0 = l->r; g.ds1 = 1;
     TL_TRY(simt_gemm(g, st));
     U = Ubuf;
@@ -234,13 +293,26 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
     g.alpha1 = 1.f; g.D = V; g.d_dt = TEMPLORA_F32; g.ds0 = l->r; g.ds1 = 1;
     TL_TRY(simt_gemm(g, st));
   }
-  if (dX) {  // dX = dY W0 + s V A
+  if (dX && !drop.xd) {  // dX = dY W0 + s V A
     SimtGemm g{};
     g.M = T; g.N = l->d_in; g.K1 = l->d_out; g.K2 = l->r;
     g.A1 = op(dY, dt, l->d_out, 1); g.B1 = op(l->W0, dt, l->d_in, 1);
     g.A2 = op(V, TEMPLORA_F32, l->r, 1); g.B2 = op(l->A, dt, l->d_in, 1);
     g.alpha1 = 1.f; g.alpha2 = l->s; g.D = dX; g.d_dt = dt; g.ds0 = l->d_in; g.ds1 = 1;
     TL_TRY(simt_gemm(g, st));
+  }
+  if (dX && drop.xd) {  // dX = dY W0, then dX += keep * s / (1 - p) * (V A)
+    SimtGemm g{};
+    g.M = T; g.N = l->d_in; g.K1 = l->d_out;
+    g.A1 = op(dY, dt, l->d_out, 1); g.B1 = op(l->W0, dt, l->d_in, 1);
+    g.alpha1 = 1.f; g.D = dX; g.d_dt = dt; g.ds0 = l->d_in; g.ds1 = 1;
+    TL_TRY(simt_gemm(g, st));
+    SimtGemm h{};
+    h.M = T; h.N = l->d_in; h.K1 = l->r;
+    h.A1 = op(V, TEMPLORA_F32, l->r, 1); h.B1 = op(l->A, dt, l->d_in, 1);
+    h.alpha1 = (float)((double)l->s / (1.0 - (double)l->dropout_p));
+    h.D = dX; h.d_dt = dt; h.ds0 = l->d_in; h.ds1 = 1; h.accumulate = 1; h.mask = drop.mask; h.mask_pitch = drop.pitch;
+    TL_TRY(simt_gemm(h, st));
   }
   {  // dB = s dY^T U
     SimtGemm g{};
@@ -252,7 +324,7 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
   {  // dA = s V^T x
     SimtGemm g{};
     g.M = l->r; g.N = l->d_in; g.K1 = T;
-    g.A1 = op(V, TEMPLORA_F32, 1, l->r); g.B1 = op(x, dt, l->d_in, 1);
+    g.A1 = op(V, TEMPLORA_F32, 1, l->r); g.B1 = op(xb, dt, l->d_in, 1);
     g.alpha1 = l->s; g.D = dA; g.d_dt = TEMPLORA_F32; g.ds0 = l->d_in; g.ds1 = 1; g.accumulate = accumulate;
     TL_TRY(simt_gemm(g, st));
   }
@@ -482,6 +554,7 @@ struct GroupBufs {
   float *Upart[kGroup], *Vpart[kGroup], *dBpart[kGroup], *dApart[kGroup];
   __nv_bfloat16 *Us[kGroup], *Vs[kGroup];
   int su[kGroup], sv[kGroup], sb[kGroup], sa[kGroup];
+  DropBufs drop[kGroup];
 };
 
 void carve_group(const templora_linear_t *proj, int n, int T, WsAlloc &ws, GroupBufs &b) {
@@ -498,18 +571,30 @@ void carve_group(const templora_linear_t *proj, int n, int T, WsAlloc &ws, Group
     b.Vs[i] = ws.take<__nv_bfloat16>((size_t)Tr);
     b.dBpart[i] = b.sb[i] > 1 ? ws.take<float>((size_t)b.sb[i] * l->d_out * l->r) : nullptr;
     b.dApart[i] = b.sa[i] > 1 ? ws.take<float>((size_t)b.sa[i] * l->d_in * l->r) : nullptr;
+    b.drop[i] = take_drop(l, T, ws);
   }
 }
 
 templora_status_t update_group_tc(const templora_linear_t *proj, const templora_param_t *As, const templora_param_t *Bs,
                                   int n, int T, const void *const *x, const void *const *dY, void *const *y,
-                                  void *const *dX, const GroupBufs &b, DeviceStatus *status, cudaStream_t st) {
+                                  void *const *dX, const GroupBufs &b, DeviceStatus *status, uint64_t steps_taken,
+                                  cudaStream_t st) {
   TcProblem probs[2 * kGroup];
   ReduceJob jobs[2 * kGroup];
-  int np = 0, nj = 0;
+  DropoutJob drops[kGroup];
+  const void *xb[kGroup];   // what the low-rank branch reads: x, or x with this step's dropout applied
+  int np = 0, nj = 0, nd = 0;
+  for (int i = 0; i < n; ++i) {
+    xb[i] = x[i];
+    if (b.drop[i].xd) {
+      drops[nd++] = drop_job(proj + i, T, x[i], b.drop[i], steps_taken);
+      xb[i] = b.drop[i].xd;
+    }
+  }
+  if (nd) TL_TRY(dropout_apply_batch(drops, nd, st));
   for (int i = 0; i < n; ++i) {
     const long long Tr = (long long)T * proj[i].r;
-    probs[np++] = prob_U(proj + i, T, x[i], b.Upart[i], b.su[i]);
+    probs[np++] = prob_U(proj + i, T, xb[i], b.Upart[i], b.su[i]);
     probs[np++] = prob_V(proj + i, T, dY[i], b.Vpart[i], b.sv[i]);
     jobs[nj++] = ReduceJob{b.Upart[i], b.su[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Us[i]};
     jobs[nj++] = ReduceJob{b.Vpart[i], b.sv[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Vs[i]};
@@ -519,15 +604,23 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
   np = 0;
   for (int i = 0; i < n; ++i) {
     probs[np++] = prob_y(proj + i, T, x[i], b.Us[i], y[i]);
-    if (dX && dX[i]) probs[np++] = prob_dX(proj + i, T, dY[i], b.Vs[i], dX[i]);
+    if (dX && dX[i]) {
+      probs[np] = prob_dX(proj + i, T, dY[i], b.Vs[i], dX[i]);
+      if (b.drop[i].xd) probs[np].Kext = 0;   // masked rank-r term: second pass below
+      ++np;
+    }
   }
   TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, use_pairs()));
+  np = 0;
+  for (int i = 0; i < n; ++i)
+    if (dX && dX[i] && b.drop[i].xd) probs[np++] = prob_dX_dropout_term(proj + i, T, b.Vs[i], dX[i], b.drop[i]);
+  if (np) TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, 0));
   np = 0; nj = 0;
   for (int i = 0; i < n; ++i) {
     const templora_linear_t *l = proj + i;
     float *gB = const_cast<float *>(Bs[i].grad), *gA = const_cast<float *>(As[i].grad);
     probs[np++] = prob_dB(l, T, dY[i], b.Us[i], b.sb[i] > 1 ? b.dBpart[i] : gB, b.sb[i]);
-    probs[np++] = prob_dA(l, T, x[i], b.Vs[i], b.sa[i] > 1 ? b.dApart[i] : gA, b.sa[i]);
+    probs[np++] = prob_dA(l, T, xb[i], b.Vs[i], b.sa[i] > 1 ? b.dApart[i] : gA, b.sa[i]);
     const long long nb = (long long)l->d_out * l->r, na = (long long)l->d_in * l->r;
     if (b.sb[i] > 1) jobs[nj++] = ReduceJob{b.dBpart[i], b.sb[i], nb, nb, 1.f, 1.f, gB, 0, nullptr};
     if (b.sa[i] > 1) jobs[nj++] = ReduceJob{b.dApart[i], b.sa[i], na, na, 1.f, 1.f, gA, 0, nullptr};
@@ -600,14 +693,16 @@ templora_status_t update_impl(const templora_linear_t *proj, const templora_para
         carve_group(proj + g0, n, rows, a, gb);
         if (a.overflow) return TEMPLORA_ERR_WORKSPACE;
         TL_TRY(update_group_tc(proj + g0, As + g0, Bs + g0, n, rows, x + g0, dY + g0, y + g0, dX ? dX + g0 : nullptr,
-                               gb, a.status(), st));
+                               gb, a.status(), (uint64_t)step, st));
       }
     } else {
       for (int i = 0; i < n_proj; ++i) {
+        templora_linear_t li = proj[i];
+        li.dropout_offset += (uint64_t)step;   // a new mask for every optimizer step
         WsAlloc a(ws_ptr, ws_bytes);
-        TL_TRY(fwd_impl(proj + i, rows, x[i], y[i], nullptr, a, false, st));
+        TL_TRY(fwd_impl(&li, rows, x[i], y[i], nullptr, a, false, st));
         WsAlloc c(ws_ptr, ws_bytes);
-        TL_TRY(bwd_impl(proj + i, rows, x[i], dY[i], nullptr, dX ? dX[i] : nullptr, const_cast<float *>(As[i].grad),
+        TL_TRY(bwd_impl(&li, rows, x[i], dY[i], nullptr, dX ? dX[i] : nullptr, const_cast<float *>(As[i].grad),
                         const_cast<float *>(Bs[i].grad), 0, c, false, st));
       }
     }

@@ -103,7 +103,9 @@ struct SimtGemm {
   void *D;
   int32_t d_dt;
   long long ds0, ds1;
-  int accumulate;            // add to existing D (fp32 outputs only)
+  int accumulate;            // add to the existing contents of D
+  const uint8_t *mask;       // optional keep bits over D's (i, j): masked-out elements add nothing
+  long long mask_pitch;
 };
 templora_status_t simt_gemm(const SimtGemm &g, cudaStream_t st);
 
@@ -124,6 +126,21 @@ struct ReduceJob {
 };
 templora_status_t reduce_partials_batch(const ReduceJob *jobs, int n_jobs, cudaStream_t st);
 
+// ---- LoRA dropout -----------------------------------------------------------------
+// xd = x * keep / (1 - p) in the storage type of x, and the keep mask as bits: byte j of row t
+// holds elements 8j .. 8j+7 (bit i = element 8j+i), mask_pitch bytes per row.
+struct DropoutJob {
+  const void *x;
+  void *xd;
+  uint8_t *mask;
+  long long T, d_in, mask_pitch;
+  int32_t dt;
+  float p;
+  uint64_t seed, offset;
+};
+templora_status_t dropout_apply_batch(const DropoutJob *jobs, int n_jobs, cudaStream_t st);
+inline long long dropout_mask_pitch(long long d_in) { return ((d_in + 7) / 8 + 15) / 16 * 16; }
+
 // ---- AdamW --------------------------------------------------------------------
 templora_status_t adamw_launch(const templora_param_t *params, int n_params, float lr, float beta1, float beta2,
                                float eps, float wd, int64_t step, int work_bf16, cudaStream_t st);
@@ -142,6 +159,11 @@ struct TcProblem {
   int out_f32;                // 1: fp32 output, 0: bf16
   long long out_s0, out_s1;   // element (i,j) of D goes to out[i*out_s0 + j*out_s1]
   long long out_split;        // element stride between split-K partial outputs
+  // optional epilogue "add under a mask": out = out_old + keep(i, j) ? epi_scale * D(i, j) : 0
+  // (keep bits as written by dropout_apply_batch; out must be row-major, out_s1 == 1)
+  const uint8_t *epi_mask;
+  long long epi_mask_pitch;
+  float epi_scale;
 };
 constexpr int kTcMaxProblems = 16;
 // BN: tile width, one of 16, 64, 256.  cta_pairs != 0 with BN == 256 runs 256 x 256 tiles on CTA pairs.

@@ -44,6 +44,78 @@ __global__ void __launch_bounds__(kRedThreads) reduce_partials_kernel(const __gr
   }
 }
 
+// ---------------------------------------------------------------- dropout ----
+// Philox4x32-10 (Salmon et al., SC'11), written from its published definition: ten rounds of
+//   (c0, c1, c2, c3) <- (hi(M1*c2) ^ c1 ^ k0, lo(M1*c2), hi(M0*c0) ^ c3 ^ k1, lo(M0*c0))
+// with the key bumped by the Weyl constants after every round.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    k.x += 0x9E3779B9u;
+    k.y += 0xBB67AE85u;
+  }
+  return c;
+}
+
+constexpr int kMaxDropJobs = 8;
+struct DropoutBatch {
+  int n_jobs;
+  int block_start[kMaxDropJobs + 1];
+  DropoutJob job[kMaxDropJobs];
+  uint32_t threshold[kMaxDropJobs];   // dropped iff draw < threshold
+  float inv_keep[kMaxDropJobs];       // 1 / (1 - p)
+};
+constexpr int kDropThreads = 256;
+
+// One thread per group of 8 consecutive elements of a row: writes 8 values of xd and one mask byte.
+__global__ void __launch_bounds__(kDropThreads) dropout_apply_kernel(const __grid_constant__ DropoutBatch b) {
+  pdl_prologue();
+  int j = 0;
+  while (j + 1 < b.n_jobs && (int)blockIdx.x >= b.block_start[j + 1]) ++j;
+  const DropoutJob &jb = b.job[j];
+  const long long groups_per_row = (jb.d_in + 7) / 8;
+  const long long gidx = (long long)(blockIdx.x - b.block_start[j]) * kDropThreads + threadIdx.x;
+  if (gidx >= jb.T * groups_per_row) return;
+  const long long t = gidx / groups_per_row, k0 = (gidx - t * groups_per_row) * 8;
+  const uint2 key = make_uint2((uint32_t)jb.seed, (uint32_t)(jb.seed >> 32));
+  const uint32_t thr = b.threshold[j];
+  const float inv = b.inv_keep[j];
+  unsigned long long cached_q = ~0ull;
+  uint4 draw = make_uint4(0, 0, 0, 0);
+  uint32_t bits = 0;
+  float vals[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    vals[i] = 0.f;
+    const long long k = k0 + i;
+    if (k >= jb.d_in) continue;
+    const unsigned long long e = (unsigned long long)(t * jb.d_in + k), q = e >> 2;
+    if (q != cached_q) {
+      draw = philox4x32_10(make_uint4((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)jb.offset, (uint32_t)(jb.offset >> 32)), key);
+      cached_q = q;
+    }
+    const uint32_t w = (e & 3) == 0 ? draw.x : (e & 3) == 1 ? draw.y : (e & 3) == 2 ? draw.z : draw.w;
+    const bool keep = w >= thr;
+    if (keep) bits |= 1u << i;
+    const long long idx = t * jb.d_in + k;
+    const float xv = jb.dt == TEMPLORA_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(jb.x)[idx])
+                                             : reinterpret_cast<const float *>(jb.x)[idx];
+    vals[i] = keep ? xv * inv : 0.f;
+  }
+  jb.mask[t * jb.mask_pitch + (k0 >> 3)] = (uint8_t)bits;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const long long k = k0 + i;
+    if (k >= jb.d_in) break;
+    const long long idx = t * jb.d_in + k;
+    if (jb.dt == TEMPLORA_BF16) reinterpret_cast<__nv_bfloat16 *>(jb.xd)[idx] = __float2bfloat16_rn(vals[i]);
+    else reinterpret_cast<float *>(jb.xd)[idx] = vals[i];
+  }
+}
+
 // ---------------------------------------------------------------- AdamW ----
 constexpr int kMaxAdam = 64;
 struct AdamTensor {
@@ -133,6 +205,32 @@ templora_status_t reduce_partials_batch(const ReduceJob *jobs, int n_jobs, cudaS
     {
       LaunchScope scope(kKindReduce, st);
       TL_CUDA_CHECK(launch_pdl(reduce_partials_kernel, dim3(blocks), dim3(kRedThreads), 0, st, b));
+    }
+    TL_CUDA_CHECK(cudaGetLastError());
+  }
+  return TEMPLORA_OK;
+}
+
+templora_status_t dropout_apply_batch(const DropoutJob *jobs, int n_jobs, cudaStream_t st) {
+  for (int j0 = 0; j0 < n_jobs; j0 += kMaxDropJobs) {
+    DropoutBatch b;
+    b.n_jobs = (n_jobs - j0 < kMaxDropJobs) ? n_jobs - j0 : kMaxDropJobs;
+    long long blocks = 0;
+    for (int j = 0; j < b.n_jobs; ++j) {
+      const DropoutJob &jb = jobs[j0 + j];
+      if (!jb.x || !jb.xd || !jb.mask || jb.T <= 0 || jb.d_in <= 0 || !(jb.p > 0.f && jb.p < 1.f)) return TEMPLORA_ERR_INVALID_ARG;
+      b.job[j] = jb;
+      double thr = floor((double)jb.p * 4294967296.0);
+      b.threshold[j] = thr >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)thr;
+      b.inv_keep[j] = (float)(1.0 / (1.0 - (double)jb.p));
+      b.block_start[j] = (int)blocks;
+      blocks += (jb.T * ((jb.d_in + 7) / 8) + kDropThreads - 1) / kDropThreads;
+    }
+    if (blocks > 0x7fffffffLL) return TEMPLORA_ERR_UNSUPPORTED;
+    b.block_start[b.n_jobs] = (int)blocks;
+    {
+      LaunchScope scope(kKindReduce, st);
+      TL_CUDA_CHECK(launch_pdl(dropout_apply_kernel, dim3((unsigned)blocks), dim3(kDropThreads), 0, st, b));
     }
     TL_CUDA_CHECK(cudaGetLastError());
   }

@@ -74,9 +74,11 @@ __global__ void __launch_bounds__(NT) simt_gemm_kernel(const SimtGemm g) {
       int gj = n0 + tx * 4 + j;
       if (gj >= g.N) continue;
       float val = g.alpha1 * acc1[i][j] + g.alpha2 * acc2[i][j];
+      if (g.mask && !((g.mask[(long long)gi * g.mask_pitch + (gj >> 3)] >> (gj & 7)) & 1)) val = 0.f;
       long long idx = (long long)gi * g.ds0 + (long long)gj * g.ds1;
       if (g.d_dt == TEMPLORA_BF16) {
-        reinterpret_cast<__nv_bfloat16 *>(g.D)[idx] = __float2bfloat16_rn(val);
+        __nv_bfloat16 *d = reinterpret_cast<__nv_bfloat16 *>(g.D);
+        d[idx] = __float2bfloat16_rn(g.accumulate ? __bfloat162float(d[idx]) + val : val);
       } else {
         float *d = reinterpret_cast<float *>(g.D);
         d[idx] = g.accumulate ? d[idx] + val : val;

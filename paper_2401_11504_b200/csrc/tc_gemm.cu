@@ -53,6 +53,10 @@ struct alignas(64) DevProb {
   long long out_s0, out_s1, out_split;
   void *out;
   int M, N, kb_main, kb_ext, splits, m_tiles, n_tiles, item_start, a_mn, b_mn, out_f32, pad;
+  const uint8_t *epi_mask;      // "add under a mask" epilogue (dropout term of dX); nullptr = plain store
+  long long epi_mask_pitch;
+  float epi_scale;
+  int pad3;
 };
 struct DevGroup {
   DevProb p[kTcMaxProblems];
@@ -209,6 +213,32 @@ __device__ __forceinline__ void store_chunk(const DevProb &q, const uint32_t (&v
   if (row >= q.M || col0 >= q.N) return;
   const long long base = (long long)split * q.out_split + (long long)row * q.out_s0 + (long long)col0 * q.out_s1;
   const int ncol = (q.N - col0 < NV) ? q.N - col0 : NV;
+  if (q.epi_mask) {
+    // out = out_old + (keep ? epi_scale * D : 0); bf16, row-major; col0 is a multiple of 8
+    __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(q.out) + base;
+    const uint8_t *mrow = q.epi_mask + (long long)row * q.epi_mask_pitch + (col0 >> 3);
+#pragma unroll
+    for (int c = 0; c < NV; c += 8) {
+      if (c >= ncol) break;
+      const uint32_t bits = mrow[c >> 3];
+      if (c + 8 <= ncol && ((reinterpret_cast<uintptr_t>(o + c) & 15) == 0)) {
+        uint4 w = *reinterpret_cast<const uint4 *>(o + c);
+        __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&w);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 old = __bfloat1622float2(h[e]);
+          if ((bits >> (2 * e)) & 1) old.x += q.epi_scale * __uint_as_float(v[c + 2 * e]);
+          if ((bits >> (2 * e + 1)) & 1) old.y += q.epi_scale * __uint_as_float(v[c + 2 * e + 1]);
+          h[e] = __floats2bfloat162_rn(old.x, old.y);
+        }
+        *reinterpret_cast<uint4 *>(o + c) = w;
+      } else {
+        for (int e = 0; e < 8 && c + e < ncol; ++e)
+          if ((bits >> e) & 1) o[c + e] = __float2bfloat16_rn(__bfloat162float(o[c + e]) + q.epi_scale * __uint_as_float(v[c + e]));
+      }
+    }
+    return;
+  }
   if (q.out_f32) {
     float *o = reinterpret_cast<float *>(q.out) + base;
     if (q.out_s1 == 1 && ncol == NV && ((reinterpret_cast<uintptr_t>(o) & 15) == 0)) {
@@ -886,6 +916,8 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     q.item_start = items;
     q.a_mn = p.a_mn; q.b_mn = p.b_mn;
     q.out_f32 = p.out_f32; q.pad = 0;
+    q.epi_mask = p.epi_mask; q.epi_mask_pitch = p.epi_mask_pitch; q.epi_scale = p.epi_scale; q.pad3 = 0;
+    if (p.epi_mask && (p.out_f32 || p.out_s1 != 1 || BN < 32)) return TEMPLORA_ERR_UNSUPPORTED;
     q.out = p.out; q.out_s0 = p.out_s0; q.out_s1 = p.out_s1; q.out_split = p.out_split;
     long long cnt = (long long)q.m_tiles * q.n_tiles * q.splits;
     if (cnt + items > 0x3fffffff) return TEMPLORA_ERR_UNSUPPORTED;

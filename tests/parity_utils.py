@@ -38,12 +38,13 @@ def f64(t):
     return inputs.to_f64(t)
 
 
-def run_fwd_bwd(b, host, s, T, with_dX=True, save_U=True, accumulate=False):
+def run_fwd_bwd(b, host, s, T, with_dX=True, save_U=True, accumulate=False, dropout=None):
     """host: dict of CPU tensors (x, W0, A, B, dY).  Returns GPU outputs as float64 numpy."""
     dev = {k: v.cuda() for k, v in host.items()}
     d_out, d_in = host["W0"].shape
     r = host["A"].shape[0]
-    lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], s)
+    dkw = {} if dropout is None else dict(dropout_p=dropout[0], dropout_seed=dropout[1], dropout_offset=dropout[2])
+    lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], s, **dkw)
     ws = b.alloc_workspace(b.templora_workspace_bytes(lin, T))
     dt = host["x"].dtype
     y = torch.full((T, d_out), float("nan"), dtype=dt, device="cuda")
@@ -64,17 +65,21 @@ def run_fwd_bwd(b, host, s, T, with_dX=True, save_U=True, accumulate=False):
     return out
 
 
-def oracle_fwd_bwd(host, s):
+def oracle_fwd_bwd(host, s, dropout=None):
     x, W0, A, B, dY = (f64(host[k]) for k in ("x", "W0", "A", "B", "dY"))
-    y, U = orc.linear_fwd(x, W0, A, B, s)
-    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, s)
+    keep, p = None, 0.0
+    if dropout is not None:
+        p = float(np.float32(dropout[0]))        # p crosses the ABI as fp32
+        keep = orc.dropout_keep(dropout[1], dropout[2], x.shape[0], x.shape[1], p)
+    y, U = orc.linear_fwd(x, W0, A, B, s, keep, p)
+    dX, dA, dB = orc.linear_bwd(x, dY, W0, A, B, s, keep, p)
     return dict(y=y, U=U, dX=dX, dA=dA, dB=dB)
 
 
 def check_fwd_bwd(b, seed, tag, T, d_in, d_out, r, s, dtype, **kw):
     host = inputs.make_linear(seed, tag, T, d_in, d_out, r, dtype=dtype, zero_B=kw.pop("zero_B", False))
     got = run_fwd_bwd(b, host, s, T, **kw)
-    ref = oracle_fwd_bwd(host, s)
+    ref = oracle_fwd_bwd(host, s, kw.get("dropout"))
     if kw.get("accumulate"):
         ref["dA"] = ref["dA"] + 1.0
         ref["dB"] = ref["dB"] + 1.0

@@ -153,13 +153,15 @@ def run_ours(args):
     c = inputs.CONFIGS[1]
     T, r, s, projections = args.chunk, args.rank, c["s"], inputs.BLOCKS[args.model]
     batch = args.batch if args.batch else T
-    default_workload = (args.model == "llama2_7b" and T == c["T"] and r == c["r"] and batch == T and args.epochs == 1)
+    default_workload = (args.model == "llama2_7b" and T == c["T"] and r == c["r"] and batch == T and args.epochs == 1
+                        and args.dropout == 0.0)
     workload = WORKLOAD if default_workload else (
-        f"{args.model}_block: 7 LoRA projections, T={T}, batch={batch}, r={r}, s={s}, fwd+bwd+AdamW, {args.epochs} epoch(s)")
+        f"{args.model}_block: 7 LoRA projections, T={T}, batch={batch}, r={r}, s={s}, fwd+bwd+AdamW, {args.epochs} epoch(s), LoRA dropout {args.dropout}")
     hp = {k: float(v) for k, v in inputs.ADAMW.items()}
     peaks = load_peaks()
 
-    blocks = [runtime.Block(b, 0, f"r{ranks.rank}/blk{i}", projections, T, r, s, "bf16", dev) for i in range(args.blocks)]
+    blocks = [runtime.Block(b, 0, f"r{ranks.rank}/blk{i}", projections, T, r, s, "bf16", dev, dropout_p=args.dropout)
+              for i in range(args.blocks)]
     N_ROT = args.blocks
     ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(blocks[0].lins, T), dev)
     steps_taken = [0] * N_ROT
@@ -206,6 +208,8 @@ def run_ours(args):
     # one launch of the fused kernel covers one batch of rows of every projection
     launches_per_step = args.epochs * -(-T // batch)
     flops_main = main_kernel_flops(projections, T, r) * args.epochs / launches_per_step
+    if args.dropout > 0:   # the rank-r term of dX runs in its own masked pass then
+        flops_main -= sum(2 * T * r * di for _, di, _ in projections) * args.epochs / launches_per_step
     achieved = flops_main / (ms_main / n_main * 1e-3) / 1e12 if n_main else None
     sha = kernel_sha1()
     traffic = TRAFFIC["bytes_per_launch"] if (TRAFFIC["tc_gemm_sha1"] == sha and default_workload) else None
@@ -230,7 +234,7 @@ def run_ours(args):
     share_ms = e0s.elapsed_time(e1s)
     kernel_share = {}
     for name, k in (("tc_main", b.KIND_TC_MAIN), ("tc_skinny", b.KIND_TC_SKINNY), ("reduce", b.KIND_REDUCE),
-                    ("adamw", b.KIND_ADAMW)):
+                    ("adamw", b.KIND_ADAMW), ("dropout", b.KIND_DROPOUT), ("tc_dropout_term", b.KIND_TC_DROPOUT_TERM)):
         ms, _, _ = b.templora_timing_read(k, reset=True)
         kernel_share[name] = round(ms / max(share_ms, 1e-9), 4)
 
@@ -450,6 +454,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="tokens per optimizer step (default: the whole chunk)")
     ap.add_argument("--rank", type=int, default=64)
     ap.add_argument("--epochs", type=int, default=1)
+    ap.add_argument("--dropout", type=float, default=0.0, help="LoRA dropout probability (paper: 0.05; the metric's workload: 0)")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--decode-blocks", type=int, default=32, help="distinct blocks the decode measurement rotates over")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -248,7 +248,7 @@ templora_status_t templora_decode_fwd_noalloc(const templora_linear_t *lin, int3
  * every launch (which costs the timed kernel and its successor their early scheduling).  Kernel classes: 0 tensor-core GEMM
  * with 256-wide tiles (y, dX), 1 tensor-core GEMM with 64-wide tiles (U, V, dA, dB),
  * 2 tensor-core GEMM with 16-wide tiles (decode), 3 partial reduction, 4 AdamW,
- * 5 generic GEMM, 6 decode finish.  Process-wide.
+ * 5 generic GEMM, 6 decode finish, 7 dropout mask, 8 masked rank-r pass of dX.  Process-wide.
  */
 void templora_timing_enable(int32_t kind_mask);
 

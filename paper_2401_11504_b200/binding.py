@@ -25,8 +25,9 @@ EXPORTS = [
     "templora_set_stream_sm_limit",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
-KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH = range(7)
-N_KINDS = 7
+(KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
+ KIND_TC_DROPOUT_TERM) = range(9)
+N_KINDS = 9
 
 
 class LinearDesc(C.Structure):

@@ -47,7 +47,9 @@ enum KernelKind {
   kKindAdamW = 4,
   kKindSimt = 5,       // generic-shape GEMM
   kKindDecodeFinish = 6,
-  kKindCount = 7
+  kKindDropout = 7,        // dropout mask + masked copy of x
+  kKindTcDropoutTerm = 8,  // tensor-core second pass adding the masked rank-r term to dX
+  kKindCount = 9
 };
 // Construct right before a kernel launch and destroy right after it.
 class LaunchScope {

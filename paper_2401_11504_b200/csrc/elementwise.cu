@@ -83,37 +83,63 @@ __global__ void __launch_bounds__(kDropThreads) dropout_apply_kernel(const __gri
   const uint2 key = make_uint2((uint32_t)jb.seed, (uint32_t)(jb.seed >> 32));
   const uint32_t thr = b.threshold[j];
   const float inv = b.inv_keep[j];
+  const uint32_t off_lo = (uint32_t)jb.offset, off_hi = (uint32_t)(jb.offset >> 32);
+  const long long idx0 = t * jb.d_in + k0;
+  if ((jb.d_in & 7) == 0) {
+    // fast path: the 8 elements are two whole Philox blocks and one 16-byte (bf16) or 32-byte (fp32) vector
+    const unsigned long long q = (unsigned long long)idx0 >> 2;
+    const uint4 d0 = philox4x32_10(make_uint4((uint32_t)q, (uint32_t)(q >> 32), off_lo, off_hi), key);
+    const uint4 d1 = philox4x32_10(make_uint4((uint32_t)(q + 1), (uint32_t)((q + 1) >> 32), off_lo, off_hi), key);
+    const uint32_t w[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+    uint32_t bits = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) bits |= (w[i] >= thr ? 1u : 0u) << i;
+    jb.mask[t * jb.mask_pitch + (k0 >> 3)] = (uint8_t)bits;
+    if (jb.dt == TEMPLORA_BF16) {
+      uint4 v = *reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(jb.x) + idx0);
+      __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(h[e]);
+        h[e] = __floats2bfloat162_rn((bits >> (2 * e)) & 1 ? f.x * inv : 0.f, (bits >> (2 * e + 1)) & 1 ? f.y * inv : 0.f);
+      }
+      *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(jb.xd) + idx0) = v;
+    } else {
+      const float4 *src = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(jb.x) + idx0);
+      float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(jb.xd) + idx0);
+      float4 a = src[0], c = src[1];
+      a.x = bits & 1 ? a.x * inv : 0.f;  a.y = bits & 2 ? a.y * inv : 0.f;
+      a.z = bits & 4 ? a.z * inv : 0.f;  a.w = bits & 8 ? a.w * inv : 0.f;
+      c.x = bits & 16 ? c.x * inv : 0.f; c.y = bits & 32 ? c.y * inv : 0.f;
+      c.z = bits & 64 ? c.z * inv : 0.f; c.w = bits & 128 ? c.w * inv : 0.f;
+      dst[0] = a; dst[1] = c;
+    }
+    return;
+  }
+  // general path: any d_in, element by element
   unsigned long long cached_q = ~0ull;
   uint4 draw = make_uint4(0, 0, 0, 0);
   uint32_t bits = 0;
-  float vals[8];
-#pragma unroll
   for (int i = 0; i < 8; ++i) {
-    vals[i] = 0.f;
     const long long k = k0 + i;
-    if (k >= jb.d_in) continue;
-    const unsigned long long e = (unsigned long long)(t * jb.d_in + k), q = e >> 2;
+    if (k >= jb.d_in) break;
+    const unsigned long long e = (unsigned long long)(idx0 + i), q = e >> 2;
     if (q != cached_q) {
-      draw = philox4x32_10(make_uint4((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)jb.offset, (uint32_t)(jb.offset >> 32)), key);
+      draw = philox4x32_10(make_uint4((uint32_t)q, (uint32_t)(q >> 32), off_lo, off_hi), key);
       cached_q = q;
     }
     const uint32_t w = (e & 3) == 0 ? draw.x : (e & 3) == 1 ? draw.y : (e & 3) == 2 ? draw.z : draw.w;
     const bool keep = w >= thr;
     if (keep) bits |= 1u << i;
-    const long long idx = t * jb.d_in + k;
-    const float xv = jb.dt == TEMPLORA_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(jb.x)[idx])
-                                             : reinterpret_cast<const float *>(jb.x)[idx];
-    vals[i] = keep ? xv * inv : 0.f;
+    if (jb.dt == TEMPLORA_BF16) {
+      const float xv = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(jb.x)[idx0 + i]);
+      reinterpret_cast<__nv_bfloat16 *>(jb.xd)[idx0 + i] = __float2bfloat16_rn(keep ? xv * inv : 0.f);
+    } else {
+      const float xv = reinterpret_cast<const float *>(jb.x)[idx0 + i];
+      reinterpret_cast<float *>(jb.xd)[idx0 + i] = keep ? xv * inv : 0.f;
+    }
   }
   jb.mask[t * jb.mask_pitch + (k0 >> 3)] = (uint8_t)bits;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const long long k = k0 + i;
-    if (k >= jb.d_in) break;
-    const long long idx = t * jb.d_in + k;
-    if (jb.dt == TEMPLORA_BF16) reinterpret_cast<__nv_bfloat16 *>(jb.xd)[idx] = __float2bfloat16_rn(vals[i]);
-    else reinterpret_cast<float *>(jb.xd)[idx] = vals[i];
-  }
 }
 
 // ---------------------------------------------------------------- AdamW ----
@@ -229,7 +255,7 @@ templora_status_t dropout_apply_batch(const DropoutJob *jobs, int n_jobs, cudaSt
     if (blocks > 0x7fffffffLL) return TEMPLORA_ERR_UNSUPPORTED;
     b.block_start[b.n_jobs] = (int)blocks;
     {
-      LaunchScope scope(kKindReduce, st);
+      LaunchScope scope(kKindDropout, st);
       TL_CUDA_CHECK(launch_pdl(dropout_apply_kernel, dim3((unsigned)blocks), dim3(kDropThreads), 0, st, b));
     }
     TL_CUDA_CHECK(cudaGetLastError());

@@ -217,25 +217,31 @@ __device__ __forceinline__ void store_chunk(const DevProb &q, const uint32_t (&v
     // out = out_old + (keep ? epi_scale * D : 0); bf16, row-major; col0 is a multiple of 8
     __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(q.out) + base;
     const uint8_t *mrow = q.epi_mask + (long long)row * q.epi_mask_pitch + (col0 >> 3);
+    if (ncol == NV && ((reinterpret_cast<uintptr_t>(o) & 15) == 0)) {
+      // all old values of the chunk are requested before any is used: one memory round trip per chunk
+      uint4 w[NV / 8];
+      uint32_t bits = 0;
 #pragma unroll
-    for (int c = 0; c < NV; c += 8) {
-      if (c >= ncol) break;
-      const uint32_t bits = mrow[c >> 3];
-      if (c + 8 <= ncol && ((reinterpret_cast<uintptr_t>(o + c) & 15) == 0)) {
-        uint4 w = *reinterpret_cast<const uint4 *>(o + c);
-        __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&w);
+      for (int c = 0; c < NV / 8; ++c) w[c] = *reinterpret_cast<const uint4 *>(o + 8 * c);
+#pragma unroll
+      for (int c = 0; c < NV / 8; ++c) bits |= (uint32_t)mrow[c] << (8 * c);
+#pragma unroll
+      for (int c = 0; c < NV / 8; ++c) {
+        __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&w[c]);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           float2 old = __bfloat1622float2(h[e]);
-          if ((bits >> (2 * e)) & 1) old.x += q.epi_scale * __uint_as_float(v[c + 2 * e]);
-          if ((bits >> (2 * e + 1)) & 1) old.y += q.epi_scale * __uint_as_float(v[c + 2 * e + 1]);
+          if ((bits >> (8 * c + 2 * e)) & 1) old.x += q.epi_scale * __uint_as_float(v[8 * c + 2 * e]);
+          if ((bits >> (8 * c + 2 * e + 1)) & 1) old.y += q.epi_scale * __uint_as_float(v[8 * c + 2 * e + 1]);
           h[e] = __floats2bfloat162_rn(old.x, old.y);
         }
-        *reinterpret_cast<uint4 *>(o + c) = w;
-      } else {
-        for (int e = 0; e < 8 && c + e < ncol; ++e)
-          if ((bits >> e) & 1) o[c + e] = __float2bfloat16_rn(__bfloat162float(o[c + e]) + q.epi_scale * __uint_as_float(v[c + e]));
       }
+#pragma unroll
+      for (int c = 0; c < NV / 8; ++c) *reinterpret_cast<uint4 *>(o + 8 * c) = w[c];
+    } else {
+      for (int c = 0; c < ncol; ++c)
+        if ((mrow[c >> 3] >> (c & 7)) & 1)
+          o[c] = __float2bfloat16_rn(__bfloat162float(o[c]) + q.epi_scale * __uint_as_float(v[c]));
     }
     return;
   }
@@ -271,6 +277,58 @@ __device__ __forceinline__ void store_chunk(const DevProb &q, const uint32_t (&v
 #pragma unroll
       for (int c = 0; c < NV; ++c)
         if (c < ncol) o[(long long)c * q.out_s1] = __float2bfloat16_rn(__uint_as_float(v[c]));
+    }
+  }
+}
+
+// Epilogue of the masked second pass of dX, one accumulator row of BN columns per thread:
+//   dX[row, n0 + c] += keep(row, n0 + c) ? epi_scale * D[row, c] : 0
+// The old values of chunk c+1 are requested while chunk c is combined and stored, so the global
+// round trip of the read-modify-write overlaps the TMEM read and the arithmetic.
+template <int BN>
+__device__ __forceinline__ void masked_add_row(const DevProb &q, uint32_t t_row, int row, int n0) {
+  const bool in_rows = row < q.M;
+  __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(q.out) + (long long)row * q.out_s0;
+  const uint8_t *mrow = q.epi_mask + (long long)row * q.epi_mask_pitch;
+  const bool vec = in_rows && (q.out_s0 % 8 == 0) && ((reinterpret_cast<uintptr_t>(q.out) & 15) == 0);
+  uint4 nxt[4];
+  uint32_t nbits = 0;
+  auto preload = [&](int col) {
+    if (vec && col + 32 <= q.N) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) nxt[c] = *reinterpret_cast<const uint4 *>(orow + col + 8 * c);
+      nbits = *reinterpret_cast<const uint32_t *>(mrow + (col >> 3));
+    }
+  };
+  preload(n0);
+  uint32_t v[32];
+#pragma unroll 1
+  for (int c0 = 0; c0 < BN; c0 += 32) {
+    const int col = n0 + c0;
+    uint4 w[4] = {nxt[0], nxt[1], nxt[2], nxt[3]};
+    const uint32_t bits = nbits;
+    if (c0 + 32 < BN) preload(col + 32);
+    tmem_ld32(t_row + c0, v);
+    tmem_ld_wait();
+    if (!in_rows || col >= q.N) continue;
+    if (vec && col + 32 <= q.N) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&w[c]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 old = __bfloat1622float2(h[e]);
+          if ((bits >> (8 * c + 2 * e)) & 1) old.x += q.epi_scale * __uint_as_float(v[8 * c + 2 * e]);
+          if ((bits >> (8 * c + 2 * e + 1)) & 1) old.y += q.epi_scale * __uint_as_float(v[8 * c + 2 * e + 1]);
+          h[e] = __floats2bfloat162_rn(old.x, old.y);
+        }
+        *reinterpret_cast<uint4 *>(orow + col + 8 * c) = w[c];
+      }
+    } else {
+      const int ncol = (q.N - col < 32) ? q.N - col : 32;
+      for (int c = 0; c < ncol; ++c)
+        if ((mrow[(col + c) >> 3] >> ((col + c) & 7)) & 1)
+          orow[col + c] = __float2bfloat16_rn(__bfloat162float(orow[col + c]) + q.epi_scale * __uint_as_float(v[c]));
     }
   }
 }
@@ -469,11 +527,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       uint32_t v[32];
       if constexpr (BN >= 32) {
+        if (q.epi_mask && BN == 256) {
+          masked_add_row<BN>(q, t_row, row, n0);
+        } else {
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-          tmem_ld32(t_row + c0, v);
-          tmem_ld_wait();
-          store_chunk<32>(q, v, row, n0 + c0, it.split);
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            tmem_ld32(t_row + c0, v);
+            tmem_ld_wait();
+            store_chunk<32>(q, v, row, n0 + c0, it.split);
+          }
         }
       } else {
         tmem_ld16(t_row, v);
@@ -835,7 +897,8 @@ templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream
   const int sms = stream_sm_limit(st, di->sm_count);
   int grid = g.n_items < sms ? g.n_items : sms;
   {
-    LaunchScope scope(BN == 256 ? kKindTcMain : (BN == 64 ? kKindTcSkinny : kKindTcDecode), st);
+    LaunchScope scope(g.p[0].epi_mask ? kKindTcDropoutTerm
+                                       : (BN == 256 ? kKindTcMain : (BN == 64 ? kKindTcSkinny : kKindTcDecode)), st);
     TL_CUDA_CHECK(launch_pdl(tc_gemm_kernel<BN>, dim3(grid), dim3(kThreads), Cfg<BN>::kSmemBytes, st, g));
   }
   TL_CUDA_CHECK(cudaGetLastError());

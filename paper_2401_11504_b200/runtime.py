@@ -73,7 +73,7 @@ class Block:
     """One block of LoRA-augmented projections resident on a device, with optimizer state."""
 
     def __init__(self, b, seed, tag, projections, T, r, s, dtype="bf16", device="cuda", with_dX=True,
-                 shared_io=None):
+                 shared_io=None, dropout_p=0.0):
         self.T, self.r, self.s, self.dtype = T, r, s, dtype
         self.names = [p[0] for p in projections]
         self.W0, self.state, self.lins, self.A_desc, self.B_desc = [], [], [], [], []
@@ -93,7 +93,8 @@ class Block:
             bb = st["B"]["work"] if dtype == "bf16" else st["B"]["master"]
             self.W0.append(W0)
             self.state.append(st)
-            self.lins.append(b.linear_desc(W0, a, bb, s))
+            self.lins.append(b.linear_desc(W0, a, bb, s, dropout_p=dropout_p,
+                                           dropout_seed=inputs._key(seed, t, "dropout") & ((1 << 64) - 1)))
             self.A_desc.append(b.param_desc(st["A"]["master"], st["A"]["m"], st["A"]["v"], st["A"]["grad"], st["A"]["work"]))
             self.B_desc.append(b.param_desc(st["B"]["master"], st["B"]["m"], st["B"]["v"], st["B"]["grad"], st["B"]["work"]))
             if shared_io is not None:

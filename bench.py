@@ -407,8 +407,19 @@ def decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=32, reps=5):
                 b.templora_decode_block_fwd(a, ws)
 
         block_args = [b.DecodeBlockArgs(lins, [xs[l.d_in] for l in lins], [ys[l.d_out] for l in lins]) for lins in blocks]
+        # the order a real decoder block imposes: q,k,v share their input; o, then gate and up, then down
+        # each wait for the step before: four grouped calls per block
+        group_args = [[b.DecodeBlockArgs(lins[i:j], [xs[l.d_in] for l in lins[i:j]], [ys[l.d_out] for l in lins[i:j]])
+                       for i, j in ((0, 3), (3, 4), (4, 6), (6, 7))] for lins in blocks]
+
+        def sweep_groups():
+            for ga in group_args:
+                for a in ga:
+                    b.templora_decode_block_fwd(a, ws)
+
         res = {}
-        for label, sweep in (("per_projection_calls", sweep_single), ("one_call_per_block", sweep_block)):
+        for label, sweep in (("per_projection_calls", sweep_single), ("four_dependent_group_calls", sweep_groups),
+                             ("one_call_per_block", sweep_block)):
             sweep()
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -198,6 +198,15 @@ const char *templora_status_string(templora_status_t st);
 templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *code, int32_t *where);
 
 /*
+ * Failure-detection self-test (the paper has no counterpart).  Enqueues one tiny kernel that
+ * waits, the way the GEMM kernels wait for their copies, on a barrier that nothing signals.
+ * After limit_ms (1..1000) it records TEMPLORA_ERR_TIMEOUT in the status record at the head of
+ * `ws` and returns normally: templora_read_device_status then reports the code, and the stream
+ * and context stay usable.  Zero the workspace head again afterwards.
+ */
+templora_status_t templora_selftest_bounded_wait(void *ws, size_t ws_bytes, int32_t limit_ms, void *stream);
+
+/*
  * Parallelized deployment (the paper's "Further Analysis": update the module in a second process or
  * stream while generation continues, then swap it in).  Caps the number of SMs that the
  * library's persistent kernels occupy when launched on `stream`, so that a chunk update on

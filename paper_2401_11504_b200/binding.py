@@ -22,7 +22,7 @@ EXPORTS = [
     "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
     "templora_timing_enable", "templora_timing_read", "templora_decode_fwd_noalloc",
     "templora_decode_block_workspace_bytes", "templora_decode_block_fwd", "templora_update_block_batched",
-    "templora_set_stream_sm_limit",
+    "templora_set_stream_sm_limit", "templora_selftest_bounded_wait",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 (KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
@@ -73,6 +73,8 @@ def _load():
     lib.templora_update_block_batched.restype = i32
     lib.templora_update_block_batched.argtypes = [LP, PP, PP, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                                   C.POINTER(vp), i32, f32, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_selftest_bounded_wait.restype = i32
+    lib.templora_selftest_bounded_wait.argtypes = [vp, sz, i32, vp]
     lib.templora_set_stream_sm_limit.restype = i32
     lib.templora_set_stream_sm_limit.argtypes = [vp, i32]
     lib.templora_status_string.restype = C.c_char_p
@@ -287,3 +289,9 @@ def templora_decode_block_fwd(args, ws, stream=None):
 def templora_set_stream_sm_limit(stream, max_sms):
     """Cap the SMs the persistent kernels use on `stream` (0 = no cap)."""
     _check(lib.templora_set_stream_sm_limit(_stream(stream), int(max_sms)), "templora_set_stream_sm_limit")
+
+
+def templora_selftest_bounded_wait(ws, limit_ms=50, stream=None):
+    """Enqueue the wait that must run out; read the outcome with templora_read_device_status."""
+    _check(lib.templora_selftest_bounded_wait(_ptr(ws), ws.numel(), int(limit_ms), _stream(stream)),
+           "templora_selftest_bounded_wait")

@@ -918,6 +918,13 @@ templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *c
   return TEMPLORA_OK;
 }
 
+templora_status_t templora_selftest_bounded_wait(void *ws, size_t ws_bytes, int32_t limit_ms, void *stream) {
+  TL_TRY(check_ws(ws, ws_bytes));
+  if (limit_ms < 1 || limit_ms > 1000) return TEMPLORA_ERR_INVALID_ARG;
+  return tc_wait_selftest(reinterpret_cast<DeviceStatus *>(ws), (unsigned long long)limit_ms * 1000000ull,
+                          reinterpret_cast<cudaStream_t>(stream));
+}
+
 templora_status_t templora_set_stream_sm_limit(void *stream, int32_t max_sms) {
   if (max_sms < 0) return TEMPLORA_ERR_INVALID_ARG;
   tc_set_stream_sm_limit(reinterpret_cast<cudaStream_t>(stream), max_sms);

@@ -173,6 +173,7 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
                                   int cta_pairs = 0);
 bool tc_available();
 void tc_set_stream_sm_limit(cudaStream_t st, int max_sms);
+templora_status_t tc_wait_selftest(DeviceStatus *status, unsigned long long limit_ns, cudaStream_t st);
 
 // ---- workspace need of the decode-time forward alone (api.cu) -------------------
 size_t decode_workspace_need(const templora_linear_t *lin, int n);

@@ -924,6 +924,38 @@ templora_status_t launch_pair(const DevGroup &g, DeviceInfo *di, cudaStream_t st
 
 }  // namespace
 
+// ------------------------------------------------------------------ bounded-wait self-test
+// One CTA waits, with the same poll / timer / status-record steps as the GEMM kernels' waits, on an
+// mbarrier that nothing will ever arrive at.  After limit_ns it must record TEMPLORA_ERR_TIMEOUT and
+// return, leaving the context usable.
+namespace {
+__global__ void wait_selftest_kernel(DeviceStatus *st, unsigned long long limit_ns, int where) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  const uint32_t bar = smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const unsigned long long t0 = globaltimer_ns();
+    bool done = false;
+    while (!done) {
+      for (int i = 0; i < 256 && !done; ++i) done = mbar_try(bar, 0);
+      if (!done && globaltimer_ns() - t0 > limit_ns) {
+        if (atomicCAS(&st->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) st->where = where;
+        __threadfence();
+        break;
+      }
+    }
+  }
+}
+}  // namespace
+
+templora_status_t tc_wait_selftest(DeviceStatus *status, unsigned long long limit_ns, cudaStream_t st) {
+  if (!status || limit_ns == 0 || limit_ns > 1000000000ull) return TEMPLORA_ERR_INVALID_ARG;   // at most 1 s
+  wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit_ns, 900);
+  TL_CUDA_CHECK(cudaGetLastError());
+  return TEMPLORA_OK;
+}
+
 void tc_set_stream_sm_limit(cudaStream_t st, int max_sms) {
   std::lock_guard<std::mutex> lk(g_limit_mu);
   if (max_sms <= 0) g_stream_limit.erase(st); else g_stream_limit[st] = max_sms;

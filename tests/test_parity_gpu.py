@@ -331,3 +331,21 @@ def test_short_workspace_is_rejected(b):
     with pytest.raises(b.TemploraError) as e:
         b.templora_linear_fwd(lin, d["x"], y, ws)
     assert e.value.code == b.ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------ failure detection
+def test_a_wait_that_nothing_satisfies_times_out_and_the_context_survives(b):
+    import time
+    ws = b.alloc_workspace(4096)
+    t0 = time.perf_counter()
+    b.templora_selftest_bounded_wait(ws, limit_ms=50)
+    code, where = b.templora_read_device_status(ws)
+    dt = time.perf_counter() - t0
+    assert code == b.ERR_TIMEOUT and where == 900
+    assert 0.04 < dt < 2.0
+    # the stream and the context are still good: a normal call right after gives a correct result
+    ws.zero_()
+    check_fwd_bwd(b, 50, "after-timeout", 130, 256, 264, 16, 2.0, "bf16")
+    # argument checks
+    with pytest.raises(b.TemploraError):
+        b.templora_selftest_bounded_wait(ws, limit_ms=5000)

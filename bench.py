@@ -390,7 +390,8 @@ def decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=32, reps=5):
             lins.append(b.linear_desc(W0, A, B, s))
         blocks.append(lins)
     bytes_per_block = sum(inputs.decode_bytes(di, do, r) for _, di, do in projections)
-    ws_bytes = max(max(b.templora_workspace_bytes(l, 16) for l in blocks[0]), b.templora_decode_block_workspace_bytes(blocks[0]))
+    ws_bytes = max([b.templora_workspace_bytes(l, 16) for l in blocks[0]] +
+                   [b.templora_decode_block_workspace_bytes(blocks[0][i:j]) for i, j in ((0, 7), (0, 3), (3, 4), (4, 6), (6, 7))])
     ws = b.alloc_workspace(ws_bytes, dev)
     out = {}
     for n in c["decode_tokens"]:

@@ -836,7 +836,32 @@ EncodeTiledFn encode_fn() {
 }
 
 // 2-D bf16 tensor [outer][inner] with row pitch `pitch` elements; box = 64 x box_outer, 128B swizzle.
+// Encoded descriptors are kept in a per-thread table: a descriptor depends only on (address, extents,
+// pitch, box), weights and state buffers keep their addresses from call to call, and encoding is a
+// sizeable part of the host time of a small call (a decode step of one projection is ~5 us of GPU work).
+struct MapKey {
+  const void *ptr;
+  long long inner, outer, pitch;
+  int box_outer;
+  bool operator==(const MapKey &o) const {
+    return ptr == o.ptr && inner == o.inner && outer == o.outer && pitch == o.pitch && box_outer == o.box_outer;
+  }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey &k) const {
+    size_t h = reinterpret_cast<size_t>(k.ptr) * 0x9E3779B97F4A7C15ull;
+    h ^= (size_t)k.inner * 0xC2B2AE3D27D4EB4Full + (size_t)k.outer * 0x165667B19E3779F9ull + (size_t)k.pitch * 31 + (size_t)k.box_outer;
+    return h ^ (h >> 29);
+  }
+};
 bool make_map(CUtensorMap *m, const void *ptr, long long inner, long long outer, long long pitch, int box_outer) {
+  static thread_local std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+  const MapKey key{ptr, inner, outer, pitch, box_outer};
+  auto it = cache.find(key);
+  if (it != cache.end()) {
+    *m = it->second;
+    return true;
+  }
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
@@ -846,7 +871,10 @@ bool make_map(CUtensorMap *m, const void *ptr, long long inner, long long outer,
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), gdim, gstr, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  if (r != CUDA_SUCCESS) return false;
+  if (cache.size() >= 8192) cache.clear();
+  cache.emplace(key, *m);
+  return true;
 }
 
 // operand [rows = M or N][K] (mn = 0) or [K][M or N] (mn = 1)

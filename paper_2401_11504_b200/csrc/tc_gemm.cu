@@ -129,6 +129,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
       : "memory");
 }
 
+// Same load with an L2 eviction-priority hint (a 64-bit policy from createpolicy).
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -399,6 +413,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
       bool ok = true;
       int item = blockIdx.x, sslot = 0;
       uint32_t sphase = 0;
+      const uint64_t stream_policy = l2_policy_evict_first();
       while (ok) {
         if (!mbar_wait(sempty_bar(sslot), sphase ^ 1u, abort_flag, g.status, 110)) { ok = false; break; }
         sched_ring[sslot] = item;
@@ -424,7 +439,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
             const uint32_t sA = smem0 + stage * kStage + j * kSub, sB = sA + kStageA;
             if (!pa_mn) {
-              tma_load_2d(sA, ma, full_bar(stage), kel, it.m0);
+              if constexpr (BN == 16)   // decode: W0 is read exactly once; keep x, A and the split-K slabs in L2 instead
+                tma_load_2d_hint(sA, ma, full_bar(stage), kel, it.m0, stream_policy);
+              else
+                tma_load_2d(sA, ma, full_bar(stage), kel, it.m0);
             } else {
 #pragma unroll
               for (int b = 0; b < BM / 64; ++b) tma_load_2d(sA + b * 8192, ma, full_bar(stage), it.m0 + b * 64, kel);

@@ -3,6 +3,7 @@
 #include "common.cuh"
 
 #include <atomic>
+#include <utility>
 #include <vector>
 
 namespace templora {
@@ -460,6 +461,70 @@ int decode_partial_rows(int kb, long long total_kb) {
   return a > b ? a : b;
 }
 
+// Cluster size (CTAs that split the k-range of one 128-row tile) for the one-kernel decode of a group:
+// the candidate whose list schedule (items in launch order, each to the cluster that frees up first)
+// ends soonest.  An item costs a cluster of S its k-blocks per CTA plus a fixed hand-over cost (measured:
+// about five k-blocks' worth), and the launched CTAs share the memory bandwidth.  0 = none applies.
+int decode_cluster_size(const templora_linear_t *proj, int np, int n, cudaStream_t st) {
+  const int cand[2] = {2, 4};
+  int best = 0;
+  double best_t = 0.0;
+  for (int c = 0; c < 2; ++c) {
+    const int S = cand[c], clusters = tc_decode_cluster_count(S, n, st);
+    bool fits = clusters >= np;
+    for (int i = 0; i < np; ++i) fits = fits && cdiv(proj[i].d_in, 64) >= S;
+    if (!fits) continue;
+    std::vector<double> load(clusters, 0.0);
+    auto give = [&](double w) {
+      int k = 0;
+      for (int j = 1; j < clusters; ++j) if (load[j] < load[k]) k = j;
+      load[k] += w;
+    };
+    const double hand_over = 5.0;
+    for (int i = 0; i < np; ++i) give((double)cdiv(proj[i].d_in, 64) / S + hand_over);
+    int order[kDecGroup];   // the launch deals the projections with the longest k-range first
+    for (int i = 0; i < np; ++i) order[i] = i;
+    for (int i = 1; i < np; ++i)
+      for (int j = i; j > 0 && proj[order[j]].d_in > proj[order[j - 1]].d_in; --j) std::swap(order[j], order[j - 1]);
+    for (int k = 0; k < np; ++k) {
+      const templora_linear_t &l = proj[order[k]];
+      const double w = (double)(cdiv(l.d_in, 64) + cdiv(l.r, 64)) / S + hand_over;
+      for (int t = 0; t < cdiv(l.d_out, 128); ++t) give(w);
+    }
+    double span = 0.0;
+    for (double l : load) span = l > span ? l : span;
+    const double t = span * S * clusters;
+    if (best == 0 || t < best_t) { best = S; best_t = t; }
+  }
+  return best;
+}
+
+// One-kernel decode of a group: per projection a u problem (A x^T, stored as bf16(s u)) and a y problem
+// (W0 x^T with the rank-r term as extension k-blocks B (s u)^T).  su: np buffers of 16 * r bf16.
+templora_status_t decode_group_cluster(const templora_linear_t *proj, int np, int n, const void *const *x,
+                                       void *const *y, __nv_bfloat16 *const *su, int S, DeviceStatus *status,
+                                       cudaStream_t st) {
+  TcProblem p[2 * kDecGroup] = {};
+  // y problems heaviest first; u problems lead the launch
+  int order[kDecGroup];
+  for (int i = 0; i < np; ++i) order[i] = i;
+  for (int i = 1; i < np; ++i)
+    for (int j = i; j > 0 && proj[order[j]].d_in > proj[order[j - 1]].d_in; --j) std::swap(order[j], order[j - 1]);
+  for (int k = 0; k < np; ++k) {
+    const int i = order[k];
+    const templora_linear_t *l = proj + i;
+    TcProblem &u = p[k], &a = p[np + k];
+    u.M = l->r; u.N = n; u.K = l->d_in;
+    u.A = l->A; u.lda = l->d_in; u.B = x[i]; u.ldb = l->d_in;
+    u.splits = 1; u.out = su[i]; u.out_s0 = 1; u.out_s1 = l->r; u.epi_scale = l->s; u.role = 1; u.flag = k;
+    a.M = l->d_out; a.N = n; a.K = l->d_in; a.Kext = l->r;
+    a.A = l->W0; a.lda = l->d_in; a.B = x[i]; a.ldb = l->d_in;
+    a.Aext = l->B; a.ldaext = l->r; a.Bext = su[i]; a.ldbext = l->r;
+    a.splits = 1; a.out = y[i]; a.out_s0 = 1; a.out_s1 = l->d_out; a.epi_scale = 1.f; a.role = 0; a.flag = k;
+  }
+  return tc_decode_cluster(p, 2 * np, n, S, status, st);
+}
+
 // Decode-time forward of up to kDecGroup projections (all on the tensor-core path): one grouped
 // launch streams every W0 and A once, one launch finishes.
 templora_status_t decode_group_tc(const templora_linear_t *proj, int np, int n, const void *const *x, void *const *y,
@@ -471,6 +536,16 @@ templora_status_t decode_group_tc(const templora_linear_t *proj, int np, int n, 
   FinishBatch fb;
   fb.n_entries = np; fb.n_tokens = n;
   int blocks = 0, max_r = 0;
+  __nv_bfloat16 *su[kDecGroup];
+  for (int i = 0; i < np; ++i) su[i] = ws.take<__nv_bfloat16>((size_t)16 * proj[i].r);
+  if (!dry && use_pairs()) {   // kernel path 2 keeps the two-kernel form below
+    if (ws.overflow) return TEMPLORA_ERR_WORKSPACE;
+    const int S = decode_cluster_size(proj, np, n, st);
+    if (S > 0) {
+      const templora_status_t rc = decode_group_cluster(proj, np, n, x, y, su, S, ws.status(), st);
+      if (rc != TEMPLORA_ERR_UNSUPPORTED) return rc;
+    }
+  }
   for (int i = 0; i < np; ++i) {
     const templora_linear_t *l = proj + i;
     const int kb = cdiv(l->d_in, 64);

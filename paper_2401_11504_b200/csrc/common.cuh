@@ -166,11 +166,21 @@ struct TcProblem {
   const uint8_t *epi_mask;
   long long epi_mask_pitch;
   float epi_scale;
+  // tc_decode_cluster only: role 0 = y of a projection, 1 = its u = A x^T (stored as bf16(epi_scale * u));
+  // flag = the projection's index within the launch
+  int role, flag;
 };
 constexpr int kTcMaxProblems = 16;
 // BN: tile width, one of 16, 64, 256.  cta_pairs != 0 with BN == 256 runs 256 x 256 tiles on CTA pairs.
 templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st,
                                   int cta_pairs = 0);
+// Decode-time forward of several projections in one launch: clusters of cluster_size (2 or 4) CTAs split
+// the k-range of each 128-row tile and sum their partial tiles through distributed shared memory.
+// Returns TEMPLORA_ERR_UNSUPPORTED when too few clusters fit (the caller then takes the two-kernel path).
+templora_status_t tc_decode_cluster(const TcProblem *probs, int n, int n_tokens, int cluster_size, DeviceStatus *status,
+                                    cudaStream_t st);
+// Clusters of cluster_size CTAs the one-kernel decode would run on this stream now (0 = not available).
+int tc_decode_cluster_count(int cluster_size, int n_tokens, cudaStream_t st);
 bool tc_available();
 void tc_set_stream_sm_limit(cudaStream_t st, int max_sms);
 templora_status_t tc_wait_selftest(DeviceStatus *status, unsigned long long limit_ns, cudaStream_t st);

@@ -22,6 +22,7 @@
 
 #include <cuda.h>
 
+#include <atomic>
 #include <mutex>
 #include <unordered_map>
 
@@ -837,6 +838,436 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 
 }  // namespace pair
 
+// ------------------------------------------------------------------ decode in one kernel (cluster split-K)
+// The decode-time forward of up to kDclMaxProj projections in a single launch.  A cluster of S CTAs
+// owns one 128-row tile of one projection's output at a time; CTA r of the cluster streams the r-th
+// part of the tile's k-blocks of W0 (TMA, evict-first) against x and accumulates its partial tile in
+// TMEM.  The partials never leave the chip: CTAs 1 .. S-1 send theirs from registers into CTA 0's
+// shared memory (st.async, counted by an mbarrier of CTA 0), CTA 0 adds them to its own in rank order
+// (deterministic) and writes y.  The rank-r term rides in the same accumulators as extension k-blocks
+// (B tile x (s u)^T) at the end of the tile's k-block sequence.  u = A x^T is itself one more item per
+// projection (the rows of A as the streamed operand): its cluster writes s*u as bf16 to scratch and
+// raises a flag (the launch's epoch number) that the other clusters' producers check before they
+// load extension operands.  The u items are dealt first, so each is the first item of its cluster
+// and waits for nothing.  Items are handed out dynamically: CTA 0's producer draws them from a global
+// counter and writes them into every CTA's item ring.
+namespace dcl {
+
+constexpr int kSub = kStageA + 16 * BK * 2;        // one k-block: 128 x 64 of W0 + 16 x 64 of x
+// Shared memory of a CTA: the operand ring (n_stages stages of KPS k-blocks), then room for the partial
+// tiles of the S - 1 other CTAs (used in CTA 0 only, but every CTA of a launch has the same layout;
+// 16 bytes per row and four tokens), then barriers and the item ring.  The host picks KPS and n_stages
+// so that the ring is as deep as the 227 KB allow: bytes in flight are what keeps HBM busy.
+constexpr int kMaxStages = 6;
+constexpr int kSmemLimit = 227 * 1024;
+__host__ __device__ constexpr int recv_bytes(int S, int n_tokens) { return (S - 1) * 128 * 16 * ((n_tokens + 3) / 4); }
+inline int stages_that_fit(int S, int kps, int n_tokens) {
+  const int n = (kSmemLimit - 2048 - recv_bytes(S, n_tokens)) / (kps * kSub);
+  return n > kMaxStages ? kMaxStages : n;
+}
+constexpr int kTmemCols = 32;
+constexpr int kDclMaxProj = 8;
+constexpr int kRing = 8;    // items the dealer may run ahead of the slowest reader in the cluster
+
+// The launch's problems travel as a DevGroup: role (DevProb::pad) 0 = a projection's y (A-op W0, B-op x,
+// extension A-op B, B-op s*u; out = y [n, d_out] bf16), 1 = its u (A-op A, B-op x; out = s*u [n, r] bf16,
+// scale in epi_scale); DevProb::pad3 = the projection's slot among the ready flags.
+struct DclParams {
+  int n_tokens, epoch, n_stages;
+};
+
+__device__ __forceinline__ int4 ld_volatile_i4(const int *p) {
+  int4 v;
+  asm volatile("ld.volatile.global.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu(int *p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_s32(uint32_t addr, int v) {
+  asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+// Remote store of 16 bytes into a peer's shared memory; the peer's mbarrier counts the bytes as they land.
+__device__ __forceinline__ void st_async_v4(uint32_t remote_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
+                                            uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(remote_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar) : "memory");
+}
+// Arrive on a peer's barrier to say "I have finished reading" (nothing of mine needs to become visible).
+__device__ __forceinline__ void mbar_arrive_remote_plain(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_acq_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait whose success also makes a peer's earlier shared-memory stores (released at cluster scope) visible.
+__device__ __noinline__ bool mbar_wait_acq_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                   DeviceStatus *st, int where) {
+  for (int i = 0; i < 4096; ++i)
+    if (mbar_try_acq_cluster(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  while (true) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_acq_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      if (st && atomicCAS(&st->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) st->where = where;
+      __threadfence();
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+template <int S, int KPS>
+__global__ void __launch_bounds__(kThreads, 1)
+    decode_cluster_kernel(const __grid_constant__ DevGroup g, const DclParams prm) {
+  constexpr int kKps = KPS, kStage = kKps * kSub;
+  const int kStages = prm.n_stages;   // runtime: what fits beside the receive buffer
+  const int nv = (prm.n_tokens + 3) >> 2;   // 16-byte pieces of a row that carry tokens
+  const int slot_bytes = 128 * 16 * nv;     // one peer's partial tile in the receive buffer
+  const int kRecvBytes = (S - 1) * slot_bytes;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_al = smem_raw + (smem0 - smem_u32(smem_raw));
+  const uint32_t recv0 = smem0 + kStages * kStage;               // CTA 0: partial tiles of CTAs 1 .. S-1
+  const float *recv_ptr = reinterpret_cast<const float *>(smem_al + kStages * kStage);
+  const uint32_t bar0 = recv0 + kRecvBytes;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
+  const uint32_t part_full = bar0 + 8u * (2 * kMaxStages + 4);      // used in CTA 0: the peers' partials have landed
+  const uint32_t part_free = bar0 + 8u * (2 * kMaxStages + 5);      // one per peer: CTA 0 has read its last partial
+  const uint32_t drain_bar = bar0 + 8u * (2 * kMaxStages + 6);
+  auto sfull_bar = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 7 + s); };            // one per CTA
+  auto sempty_bar = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 7 + kRing + s); };  // used in CTA 0
+  uint8_t *misc = smem_al + kStages * kStage + kRecvBytes + 512;
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(misc);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(misc + 4);
+  volatile int *sched_ring = reinterpret_cast<volatile int *>(misc + 16);
+  const uint32_t ring0 = bar0 + 512 + 16;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)pair::cluster_ctarank();
+  const int cluster_id = blockIdx.x / S, n_clusters = gridDim.x / S;
+  int *flags = &g.status->pad[0];
+  // every role but CTA 0's producer takes its items from the ring: 6 per CTA
+  constexpr int kRingReaders = 6 * S - 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    mbar_init(part_full, 4);       // one lane of each epilogue warp of CTA 0 (each also announces its share of the bytes)
+    mbar_init(part_free, 4);       // one lane of each epilogue warp of CTA 0
+    mbar_init(drain_bar, 1);
+    for (int s = 0; s < kRing; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), kRingReaders); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
+                 "r"((uint32_t)kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  pair::cluster_sync_all();   // the peers' barriers are initialised before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_prologue();
+
+  // this CTA's share of an item.  The item's k-blocks are those of the streamed operand followed by the
+  // extension blocks; CTA r takes the r-th of S equal parts of that sequence: nmain streamed blocks from
+  // kb0 on, then next extension blocks from ext0 on.
+  auto share_of = [&](int item, int &p, int &m0, int &kb0, int &nmain, int &ext0, int &next) {
+    p = 0;
+    while (p + 1 < g.n_prob && item >= g.p[p + 1].item_start) ++p;
+    const DevProb &q = g.p[p];
+    m0 = (item - q.item_start) * BM;
+    const int total = q.kb_main + q.kb_ext;
+    const int t0 = (int)((long long)total * rank / S), t1 = (int)((long long)total * (rank + 1) / S);
+    kb0 = t0 < q.kb_main ? t0 : q.kb_main;
+    nmain = (t1 < q.kb_main ? t1 : q.kb_main) - kb0;
+    ext0 = t0 > q.kb_main ? t0 - q.kb_main : 0;
+    next = (t1 > q.kb_main ? t1 - q.kb_main : 0) - ext0;
+  };
+  // take the next item from this CTA's ring (written by CTA 0's producer) and hand the slot back
+  auto ring_take = [&](int &sslot, uint32_t &sphase, int where, int &item) -> bool {
+    if (!mbar_wait_acq_cluster(sfull_bar(sslot), sphase, abort_flag, g.status, where)) return false;
+    item = sched_ring[sslot];
+    return true;
+  };
+  auto ring_release = [&](int &sslot, uint32_t &sphase) {
+    mbar_arrive_remote_plain(pair::mapa_shared(sempty_bar(sslot), 0));
+    if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
+  };
+
+  if (warp == 0) {
+    // ===================== TMA producer; in CTA 0 it also deals the items =====================
+    if (lane == 0) {
+      int stage = 0, sslot = 0;
+      uint32_t phase = 0, sphase = 0;
+      long long issued = 0;
+      bool ok = true;
+      int item = cluster_id;
+      const uint64_t stream_policy = l2_policy_evict_first();
+      uint32_t ready_mask = 0;   // projections whose s*u this thread has seen complete
+      // CTA 0: write an item into every CTA's ring (the slot must have been handed back by all its readers)
+      auto deal = [&](int it) -> bool {
+        if (!mbar_wait(sempty_bar(sslot), sphase ^ 1u, abort_flag, g.status, 830)) return false;
+#pragma unroll
+        for (int r = 0; r < S; ++r) st_cluster_s32(pair::mapa_shared(ring0 + 4u * sslot, (uint32_t)r), it);
+#pragma unroll
+        for (int r = 0; r < S; ++r)   // release at cluster scope: the store above is visible to whoever sees this arrival
+          pair::mbar_arrive_cluster(pair::mapa_shared(sfull_bar(sslot), (uint32_t)r));
+        if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
+        return true;
+      };
+      if (rank == 0) ok = deal(item);
+      while (ok) {
+        int next_item = 0;
+        if (rank == 0) {
+          if (item >= g.n_items) break;   // the end marker has been passed on
+          // the peers learn the next item before this CTA starts loading the current one
+          next_item = n_clusters + atomicAdd(&g.status->sched_next, 1);
+          if (!deal(next_item)) { ok = false; break; }
+        } else {
+          if (!ring_take(sslot, sphase, 831, item)) { ok = false; break; }
+          ring_release(sslot, sphase);
+          if (item >= g.n_items) break;
+        }
+        int p, m0, kb0, nmain, ext0, next;
+        share_of(item, p, m0, kb0, nmain, ext0, next);
+        const DevProb &q = g.p[p];
+        const int nkb = nmain + next;
+        bool u_ready = (next == 0) || ((ready_mask >> q.pad3) & 1u);
+        for (int i0 = 0; ok && i0 < nkb; i0 += kKps) {
+          const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
+          if (!u_ready && i0 + cnt > nmain) {
+            // s*u of this projection must be complete (another cluster writes it): bounded wait on its flag.
+            // One pass reads the flags of all projections, so each is usually waited for once per CTA.
+            const unsigned long long t0 = globaltimer_ns();
+            while (!((ready_mask >> q.pad3) & 1u)) {
+              const int4 f0 = ld_volatile_i4(flags), f1 = ld_volatile_i4(flags + 4);
+              const int f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+#pragma unroll
+              for (int w = 0; w < 8; ++w) ready_mask |= (f[w] == prm.epoch ? 1u : 0u) << w;
+              if ((ready_mask >> q.pad3) & 1u) break;
+              if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (atomicCAS(&g.status->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) g.status->where = 801;
+                __threadfence();
+                ok = false;
+                break;
+              }
+            }
+            if (!ok) break;
+            __threadfence();       // acquire side of the flag
+            fence_async_proxy();   // those generic-proxy writes are read by the TMA loads below
+            u_ready = true;
+          }
+          if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 800)) { ok = false; break; }
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(cnt * kSub));
+          for (int j = 0; j < cnt; ++j) {
+            const int i = i0 + j;
+            const uint32_t sA = smem0 + stage * kStage + j * kSub, sB = sA + kStageA;
+            if (i < nmain) {
+              const int kel = (kb0 + i) * BK;
+              tma_load_2d_hint(sA, &q.tmA, full_bar(stage), kel, m0, stream_policy);   // read exactly once
+              tma_load_2d(sB, &q.tmB, full_bar(stage), kel, 0);
+            } else {
+              const int kel = (ext0 + i - nmain) * BK;
+              tma_load_2d(sA, &q.tmAe, full_bar(stage), kel, m0);
+              tma_load_2d(sB, &q.tmBe, full_bar(stage), kel, 0);
+            }
+          }
+          ++issued;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (rank == 0) item = next_item;
+      }
+      if (!ok) {
+        // wait (bounded) for the copies this thread still has in flight before the CTA may exit
+        long long n = issued < kStages ? issued : kStages;
+        for (long long k = 0; k < n; ++k) {
+          const long long idx = issued - 1 - k;
+          const unsigned long long t0 = globaltimer_ns();
+          while (!mbar_try(full_bar((int)(idx % kStages)), (uint32_t)((idx / kStages) & 1)) &&
+                 globaltimer_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      int stage = 0, local = 0, sslot = 0;
+      uint32_t phase = 0, sphase = 0;
+      bool ok = true;
+      const uint32_t idesc = instr_desc(16, 0, 0);
+      const uint64_t tmpl = smem_desc_template(0);
+      const uint32_t kstep = smem_desc_kstep(0);
+      while (ok) {
+        int item;
+        if (!ring_take(sslot, sphase, 812, item)) { ok = false; break; }
+        ring_release(sslot, sphase);
+        if (item >= g.n_items) break;
+        int p, m0, kb0, nmain, ext0, next;
+        share_of(item, p, m0, kb0, nmain, ext0, next);
+        const int nkb = nmain + next;
+        if (nkb == 0) continue;   // nothing of this item falls to this CTA: its epilogue parks zeros
+        const int acc = local & 1;
+        const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+        ++local;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, g.status, 810)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 16);
+        for (int i0 = 0; i0 < nkb; i0 += kKps) {
+          const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
+          if (!mbar_wait_fast(full_bar(stage), phase, abort_flag, g.status, 811)) { ok = false; break; }
+          tc_fence_after();
+          for (int j = 0; j < cnt; ++j) {
+            const uint32_t a_lo = (smem0 + stage * kStage + j * kSub) >> 4, b_lo = a_lo + (kStageA >> 4);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk)
+              tc_mma_bf16(d_tmem, tmpl | (uint64_t)(a_lo + kk * kstep), tmpl | (uint64_t)(b_lo + kk * kstep), idesc,
+                          (i0 | j | kk) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit(tfull_bar(acc));
+      }
+      if (!ok) {
+        tc_commit(drain_bar);   // let MMAs already issued finish before TMEM is released
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try(drain_bar, 0) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ===================== epilogue and in-cluster reduction (warps 2..5) =====================
+    const int quarter = warp & 3;   // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
+    const int row_in_tile = quarter * 32 + lane;
+    int local = 0, sslot = 0;
+    uint32_t sphase = 0;
+    bool ok = true;
+    for (int seq = 0; ok; ++seq) {   // seq: items this cluster has taken (phase of the part_* barriers)
+      int item;
+      ok = __all_sync(0xffffffffu, ring_take(sslot, sphase, 823, item));
+      if (!ok) break;
+      __syncwarp();
+      if (lane == 0) ring_release(sslot, sphase); else if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
+      __syncwarp();
+      if (item >= g.n_items) break;
+      int p, m0, kb0, nmain, ext0, next;
+      share_of(item, p, m0, kb0, nmain, ext0, next);
+      const DevProb &q = g.p[p];
+      uint32_t v[32];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) v[c] = 0u;
+      if (nmain + next > 0) {
+        const int acc = local & 1;
+        const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+        ++local;
+        ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, g.status, 820));
+        if (!ok) break;
+        tc_fence_after();
+        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 16), v);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        __syncwarp();
+      }
+      if (rank != 0) {
+        // send this row's partial sums into CTA 0's shared memory, once CTA 0 has read the previous ones
+        ok = __all_sync(0xffffffffu, mbar_wait(part_free, (uint32_t)(seq & 1) ^ 1u, abort_flag, g.status, 821));
+        if (!ok) break;
+        const uint32_t dst = pair::mapa_shared(recv0 + (uint32_t)((rank - 1) * slot_bytes + row_in_tile * 16 * nv), 0);
+        const uint32_t bar = pair::mapa_shared(part_full, 0);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c < nv) st_async_v4(dst + 16u * c, v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3], bar);
+        continue;
+      }
+
+      // CTA 0: wait for the S - 1 other partials and add them in rank order (deterministic)
+      if (lane == 0) mbar_arrive_expect_tx(part_full, (uint32_t)((S - 1) * 32 * 16 * nv));
+      __syncwarp();   // lane 0 must have arrived before the warp starts polling: the barrier needs that arrival
+      ok = __all_sync(0xffffffffu, mbar_wait(part_full, (uint32_t)(seq & 1), abort_flag, g.status, 822));
+      if (!ok) break;
+      float sum[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) sum[c] = __uint_as_float(v[c]);
+#pragma unroll
+      for (int r = 1; r < S; ++r) {
+        const float4 *src = reinterpret_cast<const float4 *>(recv_ptr + (r - 1) * (slot_bytes / 4) + row_in_tile * 4 * nv);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c < nv) {
+            const float4 t = src[c];
+            sum[4 * c] += t.x; sum[4 * c + 1] += t.y; sum[4 * c + 2] += t.z; sum[4 * c + 3] += t.w;
+          }
+      }
+      __syncwarp();
+      if (lane == 0) {
+#pragma unroll
+        for (int r = 1; r < S; ++r) mbar_arrive_remote_plain(pair::mapa_shared(part_free, (uint32_t)r));
+      }
+      __syncwarp();
+      const int row = m0 + row_in_tile;
+      const bool is_u = q.pad == 1;
+      if (row < q.M) {
+        __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(q.out) + row;
+        const float sc = is_u ? q.epi_scale : 1.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (i < prm.n_tokens) out[(long long)i * q.out_s1] = __float2bfloat16_rn(sc * sum[i]);
+      }
+      if (is_u) {   // publish s*u: the last of the four warps to finish its rows raises the flag
+        __threadfence();
+        fence_async_proxy();
+        __syncwarp();
+        if (lane == 0) {
+          int *arrived = flags + kDclMaxProj + q.pad3;
+          if (atomicAdd(arrived, 1) == 3) {
+            *arrived = 0;
+            __threadfence();
+            st_release_gpu(flags + q.pad3, prm.epoch);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  pair::cluster_sync_all();   // no CTA leaves while a peer may still read its partial or signal its barriers
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+  }
+  // the last cluster to finish re-arms the item counter for the next launch on this workspace
+  if (rank == 0 && threadIdx.x == 0) {
+    __threadfence();
+    const int done = atomicAdd(&g.status->sched_done, 1);
+    if (done == n_clusters - 1) {
+      g.status->sched_next = 0;
+      g.status->sched_done = 0;
+      __threadfence();
+    }
+  }
+}
+
+}  // namespace dcl
+
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -918,6 +1349,7 @@ struct DeviceInfo {
   int cc_major = 0;
   bool attr_set[3] = {false, false, false};
   bool pair_attr_set = false;
+  int dcl_clusters[4] = {};   // per decode-cluster kernel variant: clusters that fit at once (0 = not asked yet, -1 = none)
 };
 DeviceInfo *device_info() {
   static DeviceInfo info[64];
@@ -968,6 +1400,60 @@ templora_status_t launch_pair(const DevGroup &g, DeviceInfo *di, cudaStream_t st
   return TEMPLORA_OK;
 }
 
+// ---- decode in one kernel: launch ------------------------------------------------
+// Clusters of S CTAs of this kernel variant that fit on the device at once (asked once per device).
+template <int S, int KPS>
+int decode_cluster_fit(DeviceInfo *di, int slot) {
+  if (di->dcl_clusters[slot] != 0) return di->dcl_clusters[slot];
+  auto kernel = dcl::decode_cluster_kernel<S, KPS>;
+  di->dcl_clusters[slot] = -1;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dcl::kSmemLimit) != cudaSuccess) return -1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kThreads);
+  cfg.gridDim = dim3(di->sm_count / S * S);
+  cfg.dynamicSmemBytes = dcl::kSmemLimit;   // one CTA per SM whatever the exact size
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int fit = 0;
+  if (cudaOccupancyMaxActiveClusters(&fit, kernel, &cfg) != cudaSuccess || fit < 1) return -1;
+  di->dcl_clusters[slot] = fit;
+  return fit;
+}
+
+template <int S, int KPS>
+templora_status_t launch_decode_cluster(const DevGroup &g, dcl::DclParams prm, DeviceInfo *di, int slot, cudaStream_t st,
+                                        int min_clusters) {
+  auto kernel = dcl::decode_cluster_kernel<S, KPS>;
+  prm.n_stages = dcl::stages_that_fit(S, KPS, prm.n_tokens);
+  if (prm.n_stages < 2) return TEMPLORA_ERR_UNSUPPORTED;
+  int clusters = decode_cluster_fit<S, KPS>(di, slot);
+  const int cap = stream_sm_limit(st, di->sm_count) / S;
+  if (clusters > cap) clusters = cap;
+  if (clusters > g.n_items) clusters = g.n_items;
+  if (clusters < 1 || clusters < min_clusters) return TEMPLORA_ERR_UNSUPPORTED;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(clusters * S);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = prm.n_stages * KPS * dcl::kSub + dcl::recv_bytes(S, prm.n_tokens) + 2048;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  {
+    LaunchScope scope(kKindTcDecode, st);
+    TL_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kernel, g, prm));
+  }
+  TL_CUDA_CHECK(cudaGetLastError());
+  return TEMPLORA_OK;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------ bounded-wait self-test
@@ -1005,6 +1491,19 @@ templora_status_t tc_wait_selftest(DeviceStatus *status, unsigned long long limi
 void tc_set_stream_sm_limit(cudaStream_t st, int max_sms) {
   std::lock_guard<std::mutex> lk(g_limit_mu);
   if (max_sms <= 0) g_stream_limit.erase(st); else g_stream_limit[st] = max_sms;
+}
+
+int tc_decode_cluster_count(int cluster_size, int n_tokens, cudaStream_t st) {
+  DeviceInfo *di = device_info();
+  if (!di || di->cc_major != 10 || n_tokens < 1 || n_tokens > 16) return 0;
+  const bool big = dcl::stages_that_fit(cluster_size, 4, n_tokens) >= 3;
+  int fit;
+  if (cluster_size == 2) fit = big ? decode_cluster_fit<2, 4>(di, 0) : decode_cluster_fit<2, 2>(di, 1);
+  else if (cluster_size == 4) fit = big ? decode_cluster_fit<4, 4>(di, 2) : decode_cluster_fit<4, 2>(di, 3);
+  else return 0;
+  const int cap = stream_sm_limit(st, di->sm_count) / cluster_size;
+  if (fit > cap) fit = cap;
+  return fit < 0 ? 0 : fit;
 }
 
 bool tc_available() {
@@ -1080,6 +1579,71 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
   if (BN == 256) return launch<256>(g, di, 0, st);
   if (BN == 64) return launch<64>(g, di, 1, st);
   return launch<16>(g, di, 2, st);
+}
+
+// Decode-time forward of up to dcl::kDclMaxProj projections in one launch.  probs holds, for each
+// projection, its u problem (role 1) and its y problem (role 0, with the rank-r extension reading the
+// u problem's output); flag is the projection's index.  The u problems must come first.
+templora_status_t tc_decode_cluster(const TcProblem *probs, int n, int n_tokens, int cluster_size, DeviceStatus *status,
+                                    cudaStream_t st) {
+  if (n <= 0 || n > kTcMaxProblems || n_tokens < 1 || n_tokens > 16) return TEMPLORA_ERR_INVALID_ARG;
+  DeviceInfo *di = device_info();
+  if (!di || di->cc_major != 10) return TEMPLORA_ERR_UNSUPPORTED;
+  if (!status) return TEMPLORA_ERR_WORKSPACE;
+  DevGroup g;
+  g.status = status;
+  g.n_prob = n;
+  int items = 0, n_u = 0;
+  for (int i = 0; i < n; ++i) {
+    const TcProblem &p = probs[i];
+    DevProb &q = g.p[i];
+    if (p.M <= 0 || p.N != n_tokens || p.K <= 0 || p.Kext < 0 || !p.A || !p.B || !p.out) return TEMPLORA_ERR_INVALID_ARG;
+    if (p.a_mn || p.b_mn || p.out_f32 || p.out_s0 != 1 || ((p.lda | p.ldb) & 7)) return TEMPLORA_ERR_UNSUPPORTED;
+    if (p.flag < 0 || p.flag >= dcl::kDclMaxProj) return TEMPLORA_ERR_INVALID_ARG;
+    if (p.role == 1) {
+      if (n_u != i || p.Kext != 0) return TEMPLORA_ERR_INVALID_ARG;   // u problems first, no extension
+      ++n_u;
+    }
+    q.M = p.M; q.N = p.N;
+    q.kb_main = (p.K + BK - 1) / BK;
+    q.kb_ext = (p.Kext + BK - 1) / BK;
+    q.splits = 1;
+    q.m_tiles = (p.M + BM - 1) / BM;
+    q.n_tiles = 1;
+    q.item_start = items;
+    q.a_mn = 0; q.b_mn = 0; q.out_f32 = 0;
+    q.pad = p.role; q.pad3 = p.flag;
+    q.epi_mask = nullptr; q.epi_mask_pitch = 0; q.epi_scale = p.epi_scale;
+    q.out = p.out; q.out_s0 = 1; q.out_s1 = p.out_s1; q.out_split = 0;
+    items += q.m_tiles;
+    bool ok = make_operand_map(&q.tmA, p.A, p.M, p.K, p.lda, 0, BM) && make_operand_map(&q.tmB, p.B, p.N, p.K, p.ldb, 0, 16);
+    if (p.Kext > 0) {
+      if (!p.Aext || !p.Bext || ((p.ldaext | p.ldbext) & 7)) return TEMPLORA_ERR_INVALID_ARG;
+      ok = ok && make_operand_map(&q.tmAe, p.Aext, p.M, p.Kext, p.ldaext, 0, BM) &&
+           make_operand_map(&q.tmBe, p.Bext, p.N, p.Kext, p.ldbext, 0, 16);
+    } else {
+      q.tmAe = q.tmA;
+      q.tmBe = q.tmB;
+    }
+    if (!ok) return TEMPLORA_ERR_CUDA;
+  }
+  g.n_items = items;
+  static std::atomic<int> epoch_counter{0};
+  dcl::DclParams prm;
+  prm.n_tokens = n_tokens;
+  do { prm.epoch = epoch_counter.fetch_add(1) + 1; } while (prm.epoch == 0);
+  // every u item must be the first item of its cluster (it then waits for nothing): the launchers
+  // below start cluster c on item c, so they need at least n_u clusters
+  // 72 KB stages (four k-blocks) when three of them fit beside the receive buffer, else 36 KB stages
+  const bool big = dcl::stages_that_fit(cluster_size, 4, n_tokens) >= 3;
+  templora_status_t rc;
+  if (cluster_size == 2)
+    rc = big ? launch_decode_cluster<2, 4>(g, prm, di, 0, st, n_u) : launch_decode_cluster<2, 2>(g, prm, di, 1, st, n_u);
+  else if (cluster_size == 4)
+    rc = big ? launch_decode_cluster<4, 4>(g, prm, di, 2, st, n_u) : launch_decode_cluster<4, 2>(g, prm, di, 3, st, n_u);
+  else
+    return TEMPLORA_ERR_INVALID_ARG;
+  return rc;
 }
 
 }  // namespace templora

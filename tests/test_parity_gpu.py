@@ -349,3 +349,45 @@ def test_a_wait_that_nothing_satisfies_times_out_and_the_context_survives(b):
     # argument checks
     with pytest.raises(b.TemploraError):
         b.templora_selftest_bounded_wait(ws, limit_ms=5000)
+
+
+# ------------------------------------------------------------------ decode: both forms, repeated calls
+def _decode_case(b, seed, tag, n, d_in, d_out, r, ws=None):
+    host = inputs.make_linear(seed, tag, n, d_in, d_out, r, dtype="bf16")
+    dev = {k: v.cuda() for k, v in host.items()}
+    lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], 2.0)
+    if ws is None:
+        ws = b.alloc_workspace(b.templora_workspace_bytes(lin, 16))
+    y = torch.full((n, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+    b.templora_decode_fwd(lin, dev["x"], y, ws)
+    assert b.templora_read_device_status(ws)[0] == 0
+    ref = orc.decode_fwd(f64(host["x"]), f64(host["W0"]), f64(host["A"]), f64(host["B"]), 2.0)
+    assert_close(f"decode y {tag}", f64(y), ref, TOL["bf16"])
+    return ws
+
+
+@pytest.mark.parametrize("n", [1, 5, 16])
+def test_decode_two_kernel_form(b, n):
+    # kernel path 2 keeps the split-K slabs + finish kernel form of the decode-time forward
+    b.templora_set_kernel_path(2)
+    try:
+        _decode_case(b, 21, f"dec2k-{n}", n, 2048, 1152, 64)
+        _decode_case(b, 21, f"dec2k-r16-{n}", n, 1000, 264, 16)
+    finally:
+        b.templora_set_kernel_path(0)
+
+
+def test_decode_repeated_calls_share_a_workspace(b):
+    # s*u of an earlier call stays in the workspace; every call must wait for its own (ready flags carry
+    # a per-launch number) and the item counter must be re-armed between calls, also across the two forms
+    d_in, d_out, r = 4096, 1280, 64
+    host = inputs.make_linear(22, "dec-rep", 16, d_in, d_out, r, dtype="bf16")
+    lin_probe = b.linear_desc(host["W0"].cuda(), host["A"].cuda(), host["B"].cuda(), 2.0)
+    ws = b.alloc_workspace(b.templora_workspace_bytes(lin_probe, 16))
+    for rep in range(6):
+        if rep == 3:
+            b.templora_set_kernel_path(2)
+        try:
+            _decode_case(b, 23 + rep, f"dec-rep-{rep}", (1, 16, 4, 7, 2, 16)[rep], d_in, d_out, r, ws=ws)
+        finally:
+            b.templora_set_kernel_path(0)

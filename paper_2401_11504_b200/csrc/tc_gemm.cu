@@ -983,20 +983,20 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t tmem_base = *tmem_slot;
   pdl_prologue();
 
-  // this CTA's share of an item.  The item's k-blocks are those of the streamed operand followed by the
-  // extension blocks; CTA r takes the r-th of S equal parts of that sequence: nmain streamed blocks from
-  // kb0 on, then next extension blocks from ext0 on.
-  auto share_of = [&](int item, int &p, int &m0, int &kb0, int &nmain, int &ext0, int &next) {
+  // this CTA's share of an item.  The streamed operand's k-blocks are dealt to the S CTAs in chunks of KPS
+  // (one pipeline stage) round-robin, so at any time the cluster reads neighbouring pieces of the same
+  // rows of W0 (the same DRAM pages): CTA r takes chunks r, r + S, ...  nmain = its streamed k-blocks.
+  // The extension blocks go to the last CTA, which never has more streamed blocks than the others.
+  auto share_of = [&](int item, int &p, int &m0, int &nmain, int &next) {
     p = 0;
     while (p + 1 < g.n_prob && item >= g.p[p + 1].item_start) ++p;
     const DevProb &q = g.p[p];
     m0 = (item - q.item_start) * BM;
-    const int total = q.kb_main + q.kb_ext;
-    const int t0 = (int)((long long)total * rank / S), t1 = (int)((long long)total * (rank + 1) / S);
-    kb0 = t0 < q.kb_main ? t0 : q.kb_main;
-    nmain = (t1 < q.kb_main ? t1 : q.kb_main) - kb0;
-    ext0 = t0 > q.kb_main ? t0 - q.kb_main : 0;
-    next = (t1 > q.kb_main ? t1 - q.kb_main : 0) - ext0;
+    const int chunks = (q.kb_main + kKps - 1) / kKps;
+    const int mine = rank < chunks ? (chunks - rank + S - 1) / S : 0;
+    nmain = mine * kKps;
+    if (mine > 0 && (chunks - 1) % S == rank) nmain -= chunks * kKps - q.kb_main;   // the ragged last chunk
+    next = (rank == S - 1) ? q.kb_ext : 0;
   };
   // take the next item from this CTA's ring (written by CTA 0's producer) and hand the slot back
   auto ring_take = [&](int &sslot, uint32_t &sphase, int where, int &item) -> bool {
@@ -1030,36 +1030,43 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
         return true;
       };
-      if (rank == 0) ok = deal(item);
+      // CTA 0 deals one item ahead (the peers learn the next item before this CTA starts loading the
+      // current one) and draws two ahead, so the counter's round trip is never waited for
+      int next_item = 0, drawn = 0;
+      if (rank == 0) {
+        next_item = n_clusters + atomicAdd(&g.status->sched_next, 1);
+        ok = deal(item);
+      }
       while (ok) {
-        int next_item = 0;
         if (rank == 0) {
           if (item >= g.n_items) break;   // the end marker has been passed on
-          // the peers learn the next item before this CTA starts loading the current one
-          next_item = n_clusters + atomicAdd(&g.status->sched_next, 1);
           if (!deal(next_item)) { ok = false; break; }
+          drawn = next_item < g.n_items ? n_clusters + atomicAdd(&g.status->sched_next, 1) : next_item;
         } else {
           if (!ring_take(sslot, sphase, 831, item)) { ok = false; break; }
           ring_release(sslot, sphase);
           if (item >= g.n_items) break;
         }
-        int p, m0, kb0, nmain, ext0, next;
-        share_of(item, p, m0, kb0, nmain, ext0, next);
+        int p, m0, nmain, next;
+        share_of(item, p, m0, nmain, next);
         const DevProb &q = g.p[p];
         const int nkb = nmain + next;
         bool u_ready = (next == 0) || ((ready_mask >> q.pad3) & 1u);
+        // the ready flags are requested now and looked at when the extension blocks come up
+        int4 f0 = make_int4(0, 0, 0, 0), f1 = f0;
+        if (!u_ready) { f0 = ld_volatile_i4(flags); f1 = ld_volatile_i4(flags + 4); }
         for (int i0 = 0; ok && i0 < nkb; i0 += kKps) {
           const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
           if (!u_ready && i0 + cnt > nmain) {
             // s*u of this projection must be complete (another cluster writes it): bounded wait on its flag.
             // One pass reads the flags of all projections, so each is usually waited for once per CTA.
             const unsigned long long t0 = globaltimer_ns();
-            while (!((ready_mask >> q.pad3) & 1u)) {
-              const int4 f0 = ld_volatile_i4(flags), f1 = ld_volatile_i4(flags + 4);
+            while (true) {
               const int f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
 #pragma unroll
               for (int w = 0; w < 8; ++w) ready_mask |= (f[w] == prm.epoch ? 1u : 0u) << w;
               if ((ready_mask >> q.pad3) & 1u) break;
+              f0 = ld_volatile_i4(flags); f1 = ld_volatile_i4(flags + 4);
               if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
                 *abort_flag = 1;
                 if (atomicCAS(&g.status->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) g.status->where = 801;
@@ -1079,11 +1086,11 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int i = i0 + j;
             const uint32_t sA = smem0 + stage * kStage + j * kSub, sB = sA + kStageA;
             if (i < nmain) {
-              const int kel = (kb0 + i) * BK;
+              const int kel = (((i / kKps) * S + rank) * kKps + i % kKps) * BK;
               tma_load_2d_hint(sA, &q.tmA, full_bar(stage), kel, m0, stream_policy);   // read exactly once
               tma_load_2d(sB, &q.tmB, full_bar(stage), kel, 0);
             } else {
-              const int kel = (ext0 + i - nmain) * BK;
+              const int kel = (i - nmain) * BK;
               tma_load_2d(sA, &q.tmAe, full_bar(stage), kel, m0);
               tma_load_2d(sB, &q.tmBe, full_bar(stage), kel, 0);
             }
@@ -1091,7 +1098,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (rank == 0) item = next_item;
+        if (rank == 0) { item = next_item; next_item = drawn; }
       }
       if (!ok) {
         // wait (bounded) for the copies this thread still has in flight before the CTA may exit
@@ -1118,8 +1125,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (!ring_take(sslot, sphase, 812, item)) { ok = false; break; }
         ring_release(sslot, sphase);
         if (item >= g.n_items) break;
-        int p, m0, kb0, nmain, ext0, next;
-        share_of(item, p, m0, kb0, nmain, ext0, next);
+        int p, m0, nmain, next;
+        share_of(item, p, m0, nmain, next);
         const int nkb = nmain + next;
         if (nkb == 0) continue;   // nothing of this item falls to this CTA: its epilogue parks zeros
         const int acc = local & 1;
@@ -1165,8 +1172,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (lane == 0) ring_release(sslot, sphase); else if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
       __syncwarp();
       if (item >= g.n_items) break;
-      int p, m0, kb0, nmain, ext0, next;
-      share_of(item, p, m0, kb0, nmain, ext0, next);
+      int p, m0, nmain, next;
+      share_of(item, p, m0, nmain, next);
       const DevProb &q = g.p[p];
       uint32_t v[32];
 #pragma unroll

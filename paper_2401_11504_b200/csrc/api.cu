@@ -3,6 +3,7 @@
 #include "common.cuh"
 
 #include <atomic>
+#include <cstring>
 #include <utility>
 #include <vector>
 
@@ -465,7 +466,28 @@ int decode_partial_rows(int kb, long long total_kb) {
 // the candidate whose list schedule (items in launch order, each to the cluster that frees up first)
 // ends soonest.  An item costs a cluster of S its k-blocks per CTA plus a fixed hand-over cost (measured:
 // about five k-blocks' worth), and the launched CTAs share the memory bandwidth.  0 = none applies.
+int decode_cluster_size_search(const templora_linear_t *proj, int np, int n, cudaStream_t st);
+// The search costs tens of microseconds of host time and a decode call only a few: the answer is
+// remembered per thread by the shapes it was found for (and by the cluster counts, which a per-stream
+// SM cap changes).
 int decode_cluster_size(const templora_linear_t *proj, int np, int n, cudaStream_t st) {
+  struct Key {
+    int np, n, c2, c4, dims[3 * kDecGroup];
+    bool operator==(const Key &o) const { return memcmp(this, &o, sizeof(Key)) == 0; }
+  };
+  static thread_local std::vector<std::pair<Key, int>> cache;
+  Key k;
+  memset(&k, 0, sizeof(k));
+  k.np = np; k.n = n; k.c2 = tc_decode_cluster_count(2, n, st); k.c4 = tc_decode_cluster_count(4, n, st);
+  for (int i = 0; i < np; ++i) { k.dims[3 * i] = proj[i].d_in; k.dims[3 * i + 1] = proj[i].d_out; k.dims[3 * i + 2] = proj[i].r; }
+  for (const auto &e : cache)
+    if (e.first == k) return e.second;
+  const int S = decode_cluster_size_search(proj, np, n, st);
+  if (cache.size() >= 256) cache.clear();
+  cache.emplace_back(k, S);
+  return S;
+}
+int decode_cluster_size_search(const templora_linear_t *proj, int np, int n, cudaStream_t st) {
   const int cand[2] = {2, 4};
   int best = 0;
   double best_t = 0.0;

@@ -219,7 +219,9 @@ templora_status_t templora_set_stream_sm_limit(void *stream, int32_t max_sms);
 /*
  * Kernel-path selection for testing: 0 = automatic (tensor-core path when the
  * shape allows, frozen-weight GEMMs on CTA pairs), 1 = always the generic kernel path,
- * 2 = tensor-core path with single-CTA tiles only.  Returns the previous value.
+ * 2 = tensor-core path with single-CTA tiles only (decode then runs as a W0 stream with
+ * split-K partials in the workspace plus a finishing kernel instead of the one-kernel cluster
+ * form).  Returns the previous value.
  * Process-wide; not part of the method.
  */
 int32_t templora_set_kernel_path(int32_t mode);
@@ -230,7 +232,7 @@ int32_t templora_set_kernel_path(int32_t mode);
  * only input and output buffers and may not call cudaMalloc themselves: a serving loop whose
  * device memory belongs entirely to another framework's pool, a latency-critical thread for
  * which an allocation (which may synchronise the device) is off limits, a plug-in without an
- * allocator.  This variant takes no workspace.  Its split-K scratch is a fixed array of
+ * allocator.  This variant takes no workspace.  Its scratch is a fixed array of
  * TEMPLORA_NOALLOC_SCRATCH_BYTES inside the library image, present on every GPU that loads
  * the library for the life of the process.  The call allocates and frees nothing.
  *   - Same arguments and result as templora_decode_fwd, minus the workspace.

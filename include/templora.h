@@ -187,6 +187,27 @@ templora_status_t templora_update_block_batched(const templora_linear_t *proj, c
                                                 float beta1, float beta2, float eps, float weight_decay,
                                                 int64_t *step_inout, void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * Linear learning-rate warm-up ("Setup": the rate is warmed up linearly over the first two
+ * chunks).  Rate of optimizer step `step` (1-based, counted over the whole run):
+ * lr * min(1, step / warmup_steps); warmup_steps <= 0 gives lr.  For the paper's setting pass
+ * warmup_steps = 2 * epochs * ceil(chunk / batch).  Host function, no GPU work.
+ */
+float templora_lr_at_step(float lr, int64_t step, int64_t warmup_steps);
+
+/*
+ * templora_update_block_batched with that warm-up applied inside the call: the optimizer step
+ * numbered k = *step_inout + 1, + 2, ... uses templora_lr_at_step(lr, k, warmup_steps).
+ * warmup_steps = 0 is templora_update_block_batched.
+ */
+templora_status_t templora_update_block_warmup(const templora_linear_t *proj, const templora_param_t *A_state,
+                                               const templora_param_t *B_state, int32_t n_proj, int32_t T,
+                                               int32_t batch_tokens, const void *const *x, const void *const *dY,
+                                               void *const *y, void *const *dX, int32_t epochs, float lr,
+                                               int64_t warmup_steps, float beta1, float beta2, float eps,
+                                               float weight_decay, int64_t *step_inout, void *ws, size_t ws_bytes,
+                                               void *stream);
+
 /* Static description of a status code. */
 const char *templora_status_string(templora_status_t st);
 

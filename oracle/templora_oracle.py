@@ -167,8 +167,18 @@ def round_bf16(a):
 # the whole update of one block of projections: n epochs over the chunk,
 # one optimizer step per epoch (batch = chunk)
 # --------------------------------------------------------------------------
+def lr_at_step(lr, step, warmup_steps):
+    """Linear learning-rate warm-up ("Setup": the rate is warmed up linearly over the first two
+    chunks): optimizer step `step` (1-based, counted over the whole run) uses
+    lr * min(1, step / warmup_steps); warmup_steps <= 0 means a constant rate.  With E epochs and
+    chunk/batch optimizer steps per epoch the paper's two chunks are warmup_steps = 2 * E * chunk/batch."""
+    if warmup_steps is None or warmup_steps <= 0:
+        return float(lr)
+    return float(lr) * min(1.0, float(step) / float(warmup_steps))
+
+
 def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf16_work=False, batch=None,
-                 dropout_p=0.0):
+                 dropout_p=0.0, warmup_steps=0, lr_round=None):
     """projs: list of dicts with keys x, dY, W0, s, A_master, B_master and optionally
     mA, vA, mB, vB (default 0).  For each epoch: forward and backward of every
     projection with the current working A, B; then step += 1 and AdamW on every
@@ -180,6 +190,10 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
     slice by slice and dA, dB are the last slice's.  With dropout_p > 0 every optimizer step
     draws a fresh mask for its row slice: projection i uses seed projs[i]["dropout_seed"]
     and offset projs[i].get("dropout_offset", 0) + (number of steps taken before this one).
+
+    With warmup_steps > 0 the step numbered k (step0 + 1, step0 + 2, ...) uses lr_at_step(lr, k,
+    warmup_steps); lr_round, if given, is applied to that rate (the tests pass the fp32 rounding
+    that the C ABI's float argument imposes).
 
     Returns (state, step): state[i] has A_master, B_master, mA, vA, mB, vB and the
     last epoch's y, dX, dA, dB.
@@ -211,9 +225,12 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
                 q["y"][rows], _ = linear_fwd(xb, p["W0"], A, B, p["s"], keep, dropout_p)
                 q["dX"][rows], q["dA"], q["dB"] = linear_bwd(xb, dYb, p["W0"], A, B, p["s"], keep, dropout_p)
             step += 1
+            lr_k = lr_at_step(lr, step, warmup_steps)
+            if lr_round is not None:
+                lr_k = lr_round(lr_k)
             for q in st:
                 q["A_master"], q["mA"], q["vA"] = adamw_step(q["A_master"], q["dA"], q["mA"], q["vA"],
-                                                             lr, beta1, beta2, eps, weight_decay, step)
+                                                             lr_k, beta1, beta2, eps, weight_decay, step)
                 q["B_master"], q["mB"], q["vB"] = adamw_step(q["B_master"], q["dB"], q["mB"], q["vB"],
-                                                             lr, beta1, beta2, eps, weight_decay, step)
+                                                             lr_k, beta1, beta2, eps, weight_decay, step)
     return st, step

@@ -22,7 +22,8 @@ EXPORTS = [
     "templora_status_string", "templora_read_device_status", "templora_set_kernel_path",
     "templora_timing_enable", "templora_timing_read", "templora_decode_fwd_noalloc",
     "templora_decode_block_workspace_bytes", "templora_decode_block_fwd", "templora_update_block_batched",
-    "templora_set_stream_sm_limit", "templora_selftest_bounded_wait",
+    "templora_set_stream_sm_limit", "templora_selftest_bounded_wait", "templora_lr_at_step",
+    "templora_update_block_warmup",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 (KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
@@ -73,6 +74,11 @@ def _load():
     lib.templora_update_block_batched.restype = i32
     lib.templora_update_block_batched.argtypes = [LP, PP, PP, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                                   C.POINTER(vp), i32, f32, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_update_block_warmup.restype = i32
+    lib.templora_update_block_warmup.argtypes = [LP, PP, PP, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                                 C.POINTER(vp), i32, f32, i64, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_lr_at_step.restype = f32
+    lib.templora_lr_at_step.argtypes = [f32, i64, i64]
     lib.templora_selftest_bounded_wait.restype = i32
     lib.templora_selftest_bounded_wait.argtypes = [vp, sz, i32, vp]
     lib.templora_set_stream_sm_limit.restype = i32
@@ -222,6 +228,21 @@ def templora_update_block_batched(args, batch_tokens, epochs, lr, beta1, beta2, 
                                              weight_decay, C.byref(st), _ptr(ws), ws.numel(), _stream(stream)),
            "templora_update_block_batched")
     return st.value
+
+
+def templora_update_block_warmup(args, batch_tokens, epochs, lr, warmup_steps, beta1, beta2, eps, weight_decay, step, ws,
+                                 stream=None):
+    """Batched chunk update with the linear learning-rate warm-up applied per optimizer step."""
+    st = C.c_int64(int(step))
+    _check(lib.templora_update_block_warmup(args.lins, args.A, args.B, args.n, args.T, int(batch_tokens), args.x,
+                                            args.dY, args.y, args.dX, int(epochs), lr, int(warmup_steps), beta1, beta2,
+                                            eps, weight_decay, C.byref(st), _ptr(ws), ws.numel(), _stream(stream)),
+           "templora_update_block_warmup")
+    return st.value
+
+
+def templora_lr_at_step(lr, step, warmup_steps):
+    return float(lib.templora_lr_at_step(lr, int(step), int(warmup_steps)))
 
 
 def templora_read_device_status(ws, stream=None):

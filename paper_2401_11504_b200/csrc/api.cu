@@ -733,7 +733,7 @@ templora_status_t update_impl(const templora_linear_t *proj, const templora_para
                               int n_proj, int T_chunk, int batch, const void *const *x_chunk,
                               const void *const *dY_chunk, void *const *y_chunk, void *const *dX_chunk, int epochs,
                               float lr, float b1, float b2, float eps, float wd, int64_t *step_inout, void *ws_ptr,
-                              size_t ws_bytes, bool dry, size_t *need, cudaStream_t st) {
+                              size_t ws_bytes, bool dry, size_t *need, cudaStream_t st, int64_t warmup_steps = 0) {
   const int T = (batch <= 0 || batch > T_chunk) ? T_chunk : batch;   // rows of a full slice
   bool all_tc = true;
   for (int i = 0; i < n_proj; ++i) all_tc = all_tc && use_tc(proj + i, dry);
@@ -804,7 +804,8 @@ templora_status_t update_impl(const templora_linear_t *proj, const templora_para
       }
     }
     ++step;
-    TL_TRY(adamw_launch(all.data(), (int)all.size(), lr, b1, b2, eps, wd, step, work_bf16, st));
+    TL_TRY(adamw_launch(all.data(), (int)all.size(), templora_lr_at_step(lr, step, warmup_steps), b1, b2, eps, wd, step,
+                        work_bf16, st));
     *step_inout = step;
   }
   return TEMPLORA_OK;
@@ -962,13 +963,30 @@ templora_status_t templora_update_block(const templora_linear_t *proj, const tem
                                        weight_decay, step_inout, ws, ws_bytes, stream);
 }
 
+float templora_lr_at_step(float lr, int64_t step, int64_t warmup_steps) {
+  if (warmup_steps <= 0 || step >= warmup_steps) return lr;
+  if (step < 0) step = 0;
+  return (float)((double)lr * ((double)step / (double)warmup_steps));
+}
+
 templora_status_t templora_update_block_batched(const templora_linear_t *proj, const templora_param_t *A_state,
                                                 const templora_param_t *B_state, int32_t n_proj, int32_t T,
                                                 int32_t batch_tokens, const void *const *x, const void *const *dY,
                                                 void *const *y, void *const *dX, int32_t epochs, float lr,
                                                 float beta1, float beta2, float eps, float weight_decay,
                                                 int64_t *step_inout, void *ws, size_t ws_bytes, void *stream) {
-  if (batch_tokens < 1) return TEMPLORA_ERR_INVALID_ARG;
+  return templora_update_block_warmup(proj, A_state, B_state, n_proj, T, batch_tokens, x, dY, y, dX, epochs, lr, 0, beta1,
+                                      beta2, eps, weight_decay, step_inout, ws, ws_bytes, stream);
+}
+
+templora_status_t templora_update_block_warmup(const templora_linear_t *proj, const templora_param_t *A_state,
+                                               const templora_param_t *B_state, int32_t n_proj, int32_t T,
+                                               int32_t batch_tokens, const void *const *x, const void *const *dY,
+                                               void *const *y, void *const *dX, int32_t epochs, float lr,
+                                               int64_t warmup_steps, float beta1, float beta2, float eps,
+                                               float weight_decay, int64_t *step_inout, void *ws, size_t ws_bytes,
+                                               void *stream) {
+  if (batch_tokens < 1 || warmup_steps < 0) return TEMPLORA_ERR_INVALID_ARG;
   if (!proj || !A_state || !B_state || n_proj <= 0 || T <= 0 || !x || !dY || !y || epochs < 0 || !step_inout ||
       *step_inout < 0)
     return TEMPLORA_ERR_INVALID_ARG;
@@ -990,7 +1008,8 @@ templora_status_t templora_update_block_batched(const templora_linear_t *proj, c
   }
   TL_TRY(check_ws(ws, ws_bytes));
   return update_impl(proj, A_state, B_state, n_proj, T, batch_tokens, x, dY, y, dX, epochs, lr, beta1, beta2, eps,
-                     weight_decay, step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream));
+                     weight_decay, step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream),
+                     warmup_steps);
 }
 
 const char *templora_status_string(templora_status_t st) {

@@ -100,3 +100,13 @@ def test_update_block_rejects_unaliased_parameters(b):
 def test_kernel_path_switch_round_trips(b):
     prev = b.templora_set_kernel_path(1)
     assert b.templora_set_kernel_path(prev) == 1
+
+
+def test_lr_at_step_host_function(b):
+    # host arithmetic only: same closed form as the oracle's, in fp32
+    import numpy as np
+    from oracle import templora_oracle as orc
+    lr = float(np.float32(5e-5))
+    for step, w in ((1, 8), (4, 8), (8, 8), (9, 8), (5, 0), (0, 4)):
+        got = b.templora_lr_at_step(lr, step, w)
+        assert got == float(np.float32(orc.lr_at_step(lr, step, w)))

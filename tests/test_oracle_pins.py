@@ -443,3 +443,36 @@ def test_update_block_with_dropout_draws_a_mask_per_step():
     # and dropout changes the result
     plain, _ = orc.update_block(projs, 2, batch=4, **hp)
     assert np.abs(plain[0]["A_master"] - st[0]["A_master"]).max() > 0
+
+
+# ------------------------------------------------------------------ learning-rate warm-up
+def test_lr_warmup_closed_forms():
+    # linear from lr/w at step 1 to lr at step w, constant after; w <= 0 switches it off
+    lr, w = 5e-5, 8
+    vals = [orc.lr_at_step(lr, k, w) for k in range(1, 13)]
+    assert vals[0] == pytest.approx(lr / w, rel=1e-15)
+    assert vals[w - 1] == lr and all(v == lr for v in vals[w:])
+    diffs = np.diff(vals[:w])
+    assert np.allclose(diffs, lr / w, rtol=1e-12)
+    assert orc.lr_at_step(lr, 1, 0) == lr and orc.lr_at_step(lr, 3, -1) == lr
+
+
+def test_update_block_warmup_equals_steps_composed_by_hand():
+    # one call over 2 epochs x 2 batches with warm-up = four single-batch calls, each with its own rate
+    # and the running step count; pins which step number each rate belongs to
+    rng = np.random.default_rng(5)
+    T, d_in, d_out, r = 8, 6, 5, 2
+    p0 = dict(x=rng.normal(size=(T, d_in)), dY=rng.normal(size=(T, d_out)), W0=rng.normal(size=(d_out, d_in)), s=1.5,
+              A_master=rng.normal(size=(r, d_in)), B_master=rng.normal(size=(d_out, r)))
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
+    ref, step = orc.update_block([p0], 2, **hp, batch=4, warmup_steps=3)
+    assert step == 4
+    cur, k = dict(p0), 0
+    for _ in range(2):
+        for rows in (slice(0, 4), slice(4, 8)):
+            q = dict(cur, x=p0["x"][rows], dY=p0["dY"][rows])
+            hp_k = dict(hp, lr=hp["lr"] * min(1.0, (k + 1) / 3.0))
+            out, k = orc.update_block([q], 1, **hp_k, step0=k)
+            cur.update({n: out[0][n] for n in ("A_master", "B_master", "mA", "vA", "mB", "vB")})
+    for n in ("A_master", "B_master", "mA", "vA", "mB", "vB"):
+        assert np.allclose(ref[0][n], cur[n], rtol=1e-13, atol=1e-15), n

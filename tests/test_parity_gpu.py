@@ -204,7 +204,7 @@ def test_adamw_many_tensors_one_call(b):
 
 
 # ------------------------------------------------------------------ update_block
-def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True, batch=None):
+def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True, batch=None, warmup=0):
     hp = hp32(hp)
     hosts = [inputs.make_linear(seed, f"ub{i}", T, di, do, r, dtype=dtype) for i, (di, do) in enumerate(shapes)]
     devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
@@ -221,7 +221,10 @@ def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True
     ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(lins, T))
     args = b.UpdateBlockArgs(lins, As, Bs, [d["x"] for d in devs], [d["dY"] for d in devs], ys,
                              dXs if with_dX else None)
-    if batch is None:
+    if warmup:
+        step = b.templora_update_block_warmup(args, batch or T, epochs, hp["lr"], warmup, hp["beta1"], hp["beta2"],
+                                              hp["eps"], hp["weight_decay"], 0, ws)
+    elif batch is None:
         step = b.templora_update_block(args, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
                                        hp["weight_decay"], 0, ws)
     else:
@@ -233,7 +236,8 @@ def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True
     projs = [dict(x=f64(h["x"]), dY=f64(h["dY"]), W0=f64(h["W0"]), s=s, A_master=f64(h["A"]), B_master=f64(h["B"]))
              for h in hosts]
     ref, rstep = orc.update_block(projs, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
-                                  bf16_work=(dtype == "bf16"), batch=batch)
+                                  bf16_work=(dtype == "bf16"), batch=batch, warmup_steps=warmup,
+                                  lr_round=lambda v: float(np.float32(v)))
     assert rstep == step
     epochs = n_steps   # below, "epochs" bounds the number of optimizer steps taken
     tol = TOL[dtype]
@@ -299,6 +303,16 @@ def test_update_block_batched_bf16(b, T, batch):
     shapes = [(256, 384), (384, 256), (256, 256)]
     _update_block_case(b, "bf16", shapes, T, 64, 2.0, 2, dict(lr=2e-4, beta1=0.9, beta2=0.999, eps=1e-8,
                                                                weight_decay=0.0), 26, batch=batch)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_update_block_with_lr_warmup(b, dtype):
+    # six optimizer steps (2 epochs x 3 batches), the rate rising linearly over the first four
+    shapes = [(256, 384), (384, 256)] if dtype == "bf16" else [(96, 80), (80, 64)]
+    r = 64 if dtype == "bf16" else 8
+    _update_block_case(b, dtype, shapes, 384 if dtype == "bf16" else 90, r, 2.0, 2,
+                       dict(lr=2e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01), 28,
+                       batch=128 if dtype == "bf16" else 30, warmup=4)
 
 
 def test_update_block_batched_fp32(b):

@@ -33,6 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel (bytes), from an ncu capture summarised under
 # profiles/; valid only while the kernel source is the one that was profiled.
+SHARED_INPUTS = [["q", "k", "v"], ["gate", "up"]]   # projections of a decoder block that read the same tensor
 TRAFFIC = {"tc_gemm_sha1": "2adce7a4be89190307bd16910780a2efe7dbf3bf", "bytes_per_launch": 1356845608}
 
 
@@ -154,9 +155,10 @@ def run_ours(args):
     T, r, s, projections = args.chunk, args.rank, c["s"], inputs.BLOCKS[args.model]
     batch = args.batch if args.batch else T
     default_workload = (args.model == "llama2_7b" and T == c["T"] and r == c["r"] and batch == T and args.epochs == 1
-                        and args.dropout == 0.0)
+                        and args.dropout == 0.0 and not args.shared_input)
     workload = WORKLOAD if default_workload else (
-        f"{args.model}_block: 7 LoRA projections, T={T}, batch={batch}, r={r}, s={s}, fwd+bwd+AdamW, {args.epochs} epoch(s), LoRA dropout {args.dropout}")
+        f"{args.model}_block: 7 LoRA projections, T={T}, batch={batch}, r={r}, s={s}, fwd+bwd+AdamW, {args.epochs} epoch(s), LoRA dropout {args.dropout}"
+        + (", q,k,v and gate,up on shared inputs with summed dX" if args.shared_input else ""))
     hp = {k: float(v) for k, v in inputs.ADAMW.items()}
     peaks = load_peaks()
 
@@ -179,7 +181,8 @@ def run_ours(args):
         blocks = stack
         update_args = [stack_args]
     else:
-        blocks = [runtime.Block(b, 0, f"r{ranks.rank}/blk{i}", projections, T, r, s, "bf16", dev, dropout_p=args.dropout)
+        blocks = [runtime.Block(b, 0, f"r{ranks.rank}/blk{i}", projections, T, r, s, "bf16", dev, dropout_p=args.dropout,
+                                input_groups=SHARED_INPUTS if args.shared_input else None)
                   for i in range(args.blocks)]
         update_args = [blk.args for blk in blocks]
     N_ROT = len(update_args)
@@ -498,6 +501,8 @@ def main():
     ap.add_argument("--stacked-blocks", type=int, default=0,
                     help="update this many blocks in one call (32 with --epochs 2: the full 7B-stack chunk update)")
     ap.add_argument("--dropout", type=float, default=0.0, help="LoRA dropout probability (paper: 0.05; the metric's workload: 0)")
+    ap.add_argument("--shared-input", action="store_true",
+                    help="q,k,v and gate,up read one input each and get one summed dX each (templora_linear_t.input_group)")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--decode-blocks", type=int, default=32, help="distinct blocks the decode measurement rotates over")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -72,7 +72,13 @@ typedef struct {
    * number of optimizer steps already taken, so every step draws a new mask.  The
    * decode-time forward never drops.  */
   float dropout_p;
-  int32_t reserved;
+  /* Projections that read the same input (q, k, v of one block; gate and up): give them the same
+   * nonzero input_group and the same dX buffer in templora_update_block*, and that buffer receives
+   * the SUM of their input gradients, i.e. the gradient with respect to the shared input, formed in
+   * one accumulator.  At most three projections per group, equal d_in, all within one run of eight
+   * consecutive projections starting at a multiple of eight.  0 = on its own (dX, if given, is this
+   * projection's own gradient, as in templora_linear_bwd).  Ignored by the other entry points.  */
+  int32_t input_group;
   uint64_t dropout_seed;
   uint64_t dropout_offset;
 } templora_linear_t;

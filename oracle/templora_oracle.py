@@ -191,6 +191,11 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
     draws a fresh mask for its row slice: projection i uses seed projs[i]["dropout_seed"]
     and offset projs[i].get("dropout_offset", 0) + (number of steps taken before this one).
 
+    A projection with key "dX_to" = j (an earlier projection with the same input width, typically q for k
+    and v, gate for up: projections that read the same input) adds its input gradient into projection
+    j's dX instead of keeping its own: state[j]["dX"] is then the gradient of the loss with respect to
+    the shared input, and state[i]["dX"] is that same array.
+
     With warmup_steps > 0 the step numbered k (step0 + 1, step0 + 2, ...) uses lr_at_step(lr, k,
     warmup_steps); lr_round, if given, is applied to that rate (the tests pass the fp32 rounding
     that the C ABI's float argument imposes).
@@ -223,7 +228,11 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
                     keep = dropout_keep(p["dropout_seed"], p.get("dropout_offset", 0) + step, xb.shape[0],
                                         xb.shape[1], dropout_p)
                 q["y"][rows], _ = linear_fwd(xb, p["W0"], A, B, p["s"], keep, dropout_p)
-                q["dX"][rows], q["dA"], q["dB"] = linear_bwd(xb, dYb, p["W0"], A, B, p["s"], keep, dropout_p)
+                dXb, q["dA"], q["dB"] = linear_bwd(xb, dYb, p["W0"], A, B, p["s"], keep, dropout_p)
+                if p.get("dX_to") is None:
+                    q["dX"][rows] = dXb
+                else:
+                    st[p["dX_to"]]["dX"][rows] += dXb
             step += 1
             lr_k = lr_at_step(lr, step, warmup_steps)
             if lr_round is not None:
@@ -233,4 +242,7 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
                                                              lr_k, beta1, beta2, eps, weight_decay, step)
                 q["B_master"], q["mB"], q["vB"] = adamw_step(q["B_master"], q["dB"], q["mB"], q["vB"],
                                                              lr_k, beta1, beta2, eps, weight_decay, step)
+    for p, q in zip(projs, st):
+        if p.get("dX_to") is not None:
+            q["dX"] = st[p["dX_to"]]["dX"]
     return st, step

@@ -34,7 +34,7 @@ N_KINDS = 9
 class LinearDesc(C.Structure):
     _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32), ("r", C.c_int32), ("s", C.c_float),
                 ("dtype", C.c_int32), ("W0", C.c_void_p), ("A", C.c_void_p), ("B", C.c_void_p),
-                ("dropout_p", C.c_float), ("reserved", C.c_int32), ("dropout_seed", C.c_uint64),
+                ("dropout_p", C.c_float), ("input_group", C.c_int32), ("dropout_seed", C.c_uint64),
                 ("dropout_offset", C.c_uint64)]
 
 
@@ -132,7 +132,7 @@ def dtype_code(t):
     raise TypeError(f"unsupported storage dtype {t.dtype}")
 
 
-def linear_desc(W0, A, B, s, dropout_p=0.0, dropout_seed=0, dropout_offset=0):
+def linear_desc(W0, A, B, s, dropout_p=0.0, dropout_seed=0, dropout_offset=0, input_group=0):
     """templora_linear_t for contiguous device tensors W0 [d_out,d_in], A [r,d_in], B [d_out,r]."""
     for t in (W0, A, B):
         if not t.is_contiguous():
@@ -142,7 +142,7 @@ def linear_desc(W0, A, B, s, dropout_p=0.0, dropout_seed=0, dropout_offset=0):
     if tuple(A.shape) != (r, d_in) or tuple(B.shape) != (d_out, r) or A.dtype != W0.dtype or B.dtype != W0.dtype:
         raise ValueError("shape/dtype mismatch between W0, A and B")
     desc = LinearDesc(d_in, d_out, r, float(s), dtype_code(W0), W0.data_ptr(), A.data_ptr(), B.data_ptr(),
-                      float(dropout_p), 0, int(dropout_seed), int(dropout_offset))
+                      float(dropout_p), int(input_group), int(dropout_seed), int(dropout_offset))
     desc._keep = (W0, A, B)  # the descriptor holds raw pointers: keep the tensors alive with it
     return desc
 

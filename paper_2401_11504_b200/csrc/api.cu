@@ -217,8 +217,10 @@ templora_status_t fwd_impl(const templora_linear_t *l, int T, const void *x, voi
 
 // ---------------------------------------------------------------- backward
 templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, const void *dY, const float *U_saved,
-                           void *dX, float *dA, float *dB, int accumulate, WsAlloc &ws, bool dry, cudaStream_t st) {
+                           void *dX, float *dA, float *dB, int accumulate, WsAlloc &ws, bool dry, cudaStream_t st,
+                           int dx_accumulate = 0) {
   const long long Tr = (long long)T * l->r;
+  if (dx_accumulate && use_tc(l, dry)) return TEMPLORA_ERR_UNSUPPORTED;   // summed dX: grouped path or generic kernels
   if (use_tc(l, dry)) {
     const int su = U_saved ? 1 : splits_skinny(T, l->r, l->d_in, 2);
     const int sv = splits_skinny(T, l->r, l->d_out, 2);
@@ -300,14 +302,14 @@ templora_status_t bwd_impl(const templora_linear_t *l, int T, const void *x, con
     g.M = T; g.N = l->d_in; g.K1 = l->d_out; g.K2 = l->r;
     g.A1 = op(dY, dt, l->d_out, 1); g.B1 = op(l->W0, dt, l->d_in, 1);
     g.A2 = op(V, TEMPLORA_F32, l->r, 1); g.B2 = op(l->A, dt, l->d_in, 1);
-    g.alpha1 = 1.f; g.alpha2 = l->s; g.D = dX; g.d_dt = dt; g.ds0 = l->d_in; g.ds1 = 1;
+    g.alpha1 = 1.f; g.alpha2 = l->s; g.D = dX; g.d_dt = dt; g.ds0 = l->d_in; g.ds1 = 1; g.accumulate = dx_accumulate;
     TL_TRY(simt_gemm(g, st));
   }
   if (dX && drop.xd) {  // dX = dY W0, then dX += keep * s / (1 - p) * (V A)
     SimtGemm g{};
     g.M = T; g.N = l->d_in; g.K1 = l->d_out;
     g.A1 = op(dY, dt, l->d_out, 1); g.B1 = op(l->W0, dt, l->d_in, 1);
-    g.alpha1 = 1.f; g.D = dX; g.d_dt = dt; g.ds0 = l->d_in; g.ds1 = 1;
+    g.alpha1 = 1.f; g.D = dX; g.d_dt = dt; g.ds0 = l->d_in; g.ds1 = 1; g.accumulate = dx_accumulate;
     TL_TRY(simt_gemm(g, st));
     SimtGemm h{};
     h.M = T; h.N = l->d_in; h.K1 = l->r;
@@ -699,19 +701,46 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
   TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
   TL_TRY(reduce_partials_batch(jobs, nj, st));
   np = 0;
+  // Projections given the same dX buffer (they share their input) get ONE problem: the products of the
+  // later ones are appended to the first one's k-loop, so the sum forms in the accumulator.
+  int owner[kGroup], rank_in_set[kGroup], prob_of[kGroup], max_rank = 0;
+  for (int i = 0; i < n; ++i) {
+    owner[i] = i; rank_in_set[i] = 0; prob_of[i] = -1;
+    if (!(dX && dX[i])) continue;
+    for (int k = 0; k < i && proj[i].input_group != 0; ++k)
+      if (dX[k] && proj[k].input_group == proj[i].input_group) { owner[i] = owner[k]; ++rank_in_set[i]; }
+    if (rank_in_set[i] > max_rank) max_rank = rank_in_set[i];
+  }
   for (int i = 0; i < n; ++i) {
     probs[np++] = prob_y(proj + i, T, x[i], b.Us[i], y[i]);
-    if (dX && dX[i]) {
+    if (!(dX && dX[i])) continue;
+    if (owner[i] == i) {
+      prob_of[i] = np;
       probs[np] = prob_dX(proj + i, T, dY[i], b.Vs[i], dX[i]);
       if (b.drop[i].xd) probs[np].Kext = 0;   // masked rank-r term: second pass below
       ++np;
+    } else {
+      TcProblem &o = probs[prob_of[owner[i]]];
+      if (proj[i].d_in != proj[owner[i]].d_in || o.n_extra + 2 > 4) return TEMPLORA_ERR_INVALID_ARG;
+      int e = o.n_extra;
+      o.Ax[e] = dY[i]; o.ldax[e] = proj[i].d_out; o.Bx[e] = proj[i].W0; o.ldbx[e] = proj[i].d_in; o.Kx[e] = proj[i].d_out;
+      ++e;
+      if (!b.drop[i].xd) {
+        o.Ax[e] = b.Vs[i]; o.ldax[e] = proj[i].r; o.Bx[e] = proj[i].A; o.ldbx[e] = proj[i].d_in; o.Kx[e] = proj[i].r;
+        ++e;
+      }
+      o.n_extra = e;
     }
   }
   TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, use_pairs()));
-  np = 0;
-  for (int i = 0; i < n; ++i)
-    if (dX && dX[i] && b.drop[i].xd) probs[np++] = prob_dX_dropout_term(proj + i, T, b.Vs[i], dX[i], b.drop[i]);
-  if (np) TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, 0));
+  // masked rank-r terms: read-modify-write passes; those aimed at the same buffer go in successive launches
+  for (int round = 0; round <= max_rank; ++round) {
+    np = 0;
+    for (int i = 0; i < n; ++i)
+      if (dX && dX[i] && b.drop[i].xd && rank_in_set[i] == round)
+        probs[np++] = prob_dX_dropout_term(proj + i, T, b.Vs[i], dX[i], b.drop[i]);
+    if (np) TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, 0));
+  }
   np = 0; nj = 0;
   for (int i = 0; i < n; ++i) {
     const templora_linear_t *l = proj + i;
@@ -799,8 +828,16 @@ templora_status_t update_impl(const templora_linear_t *proj, const templora_para
         WsAlloc a(ws_ptr, ws_bytes);
         TL_TRY(fwd_impl(&li, rows, x[i], y[i], nullptr, a, false, st));
         WsAlloc c(ws_ptr, ws_bytes);
-        TL_TRY(bwd_impl(&li, rows, x[i], dY[i], nullptr, dX ? dX[i] : nullptr, const_cast<float *>(As[i].grad),
-                        const_cast<float *>(Bs[i].grad), 0, c, false, st));
+        int shared_before = 0;   // an earlier projection of this step wrote the same dX: add to it
+        for (int k = i - i % kGroup; k < i && dX && dX[i] && proj[i].input_group != 0; ++k)
+          shared_before += (dX[k] && proj[k].input_group == proj[i].input_group) ? 1 : 0;
+        const int saved_override = t_path_override;
+        if (shared_before) t_path_override = 1;   // the generic kernels can accumulate into dX
+        const templora_status_t rc =
+            bwd_impl(&li, rows, x[i], dY[i], nullptr, dX ? dX[i] : nullptr, const_cast<float *>(As[i].grad),
+                     const_cast<float *>(Bs[i].grad), 0, c, false, st, shared_before ? 1 : 0);
+        t_path_override = saved_override;
+        TL_TRY(rc);
       }
     }
     ++step;
@@ -997,6 +1034,16 @@ templora_status_t templora_update_block_warmup(const templora_linear_t *proj, co
     if (proj[i].dtype != proj[0].dtype) return TEMPLORA_ERR_UNSUPPORTED;
     if (!x[i] || !dY[i] || !y[i] || !aligned16(x[i]) || !aligned16(dY[i]) || !aligned16(y[i])) return TEMPLORA_ERR_INVALID_ARG;
     if (dX && dX[i] && !aligned16(dX[i])) return TEMPLORA_ERR_INVALID_ARG;
+    if (proj[i].input_group != 0 && dX && dX[i]) {
+      // members of an input group (within one run of eight projections): one dX buffer, one input width, at most three
+      int sharers = 0;
+      for (int k = i - i % kGroup; k < i; ++k)
+        if (dX[k] && proj[k].input_group == proj[i].input_group) {
+          ++sharers;
+          if (proj[k].d_in != proj[i].d_in || dX[k] != dX[i]) return TEMPLORA_ERR_INVALID_ARG;
+        }
+      if (sharers > 2) return TEMPLORA_ERR_INVALID_ARG;
+    }
     const templora_param_t &a = A_state[i], &b = B_state[i];
     if (a.n != (int64_t)proj[i].r * proj[i].d_in || b.n != (int64_t)proj[i].d_out * proj[i].r) return TEMPLORA_ERR_INVALID_ARG;
     if (!a.master || !a.m || !a.v || !a.grad || !b.master || !b.m || !b.v || !b.grad) return TEMPLORA_ERR_INVALID_ARG;

@@ -166,6 +166,13 @@ struct TcProblem {
   const uint8_t *epi_mask;
   long long epi_mask_pitch;
   float epi_scale;
+  // further operand pairs accumulated into the same output (input gradients of projections that share
+  // their input, summed): D += Ax[e][M, Kx[e]] Bx[e][N, Kx[e]]^T, stored like A and B (same a_mn, b_mn);
+  // not with split-K
+  int n_extra;
+  const void *Ax[4], *Bx[4];
+  long long ldax[4], ldbx[4];
+  int Kx[4];
   // tc_decode_cluster only: role 0 = y of a projection, 1 = its u = A x^T (stored as bf16(epi_scale * u));
   // flag = the projection's index within the launch
   int role, flag;

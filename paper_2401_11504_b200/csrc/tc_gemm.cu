@@ -49,8 +49,11 @@ template <> struct Cfg<256> : CfgBase<256, 4, 512, 1> {};
 template <> struct Cfg<64> : CfgBase<64, 8, 128, 1> {};
 template <> struct Cfg<16> : CfgBase<16, 3, 32, 4> {};
 
+constexpr int kMaxExtra = 4;   // further operand pairs accumulated into the same output tile
 struct alignas(64) DevProb {
   CUtensorMap tmA, tmB, tmAe, tmBe;
+  CUtensorMap tmXa[kMaxExtra], tmXb[kMaxExtra];
+  int kb_x[kMaxExtra], kb_xtot;   // k-blocks of each extra pair and their sum (the pairs follow the extension)
   long long out_s0, out_s1, out_split;
   void *out;
   int M, N, kb_main, kb_ext, splits, m_tiles, n_tiles, item_start, a_mn, b_mn, out_f32, pad;
@@ -218,9 +221,30 @@ __device__ __forceinline__ Item decode_item(const DevGroup &g, int item) {
   it.split = local / q.n_tiles;
   it.kb0 = (int)((long long)q.kb_main * it.split / q.splits);
   it.kb1 = (int)((long long)q.kb_main * (it.split + 1) / q.splits);
-  it.next = (it.split == q.splits - 1) ? q.kb_ext : 0;
+  it.next = (it.split == q.splits - 1) ? q.kb_ext + q.kb_xtot : 0;
   return it;
 }
+
+// Walks the k-blocks of a work item in order: the streamed range of the main operand pair, then the
+// extension pair, then the extra pairs.  take() yields the maps and the k element offset of the next block.
+struct KCursor {
+  const DevProb &q;
+  const CUtensorMap *ma, *mb;
+  int seg, left, kel;
+  __device__ __forceinline__ KCursor(const DevProb &q_, int kb0, int nmain)
+      : q(q_), ma(&q_.tmA), mb(&q_.tmB), seg(0), left(nmain), kel(kb0 * BK) {}
+  __device__ __forceinline__ void take(const CUtensorMap *&a, const CUtensorMap *&b, int &k) {
+    while (left == 0 && seg <= kMaxExtra) {   // the caller never asks for more blocks than the item has
+      ++seg;
+      kel = 0;
+      if (seg == 1) { ma = &q.tmAe; mb = &q.tmBe; left = q.kb_ext; }
+      else { ma = &q.tmXa[seg - 2]; mb = &q.tmXb[seg - 2]; left = q.kb_x[seg - 2]; }
+    }
+    a = ma; b = mb; k = kel;
+    kel += BK;
+    --left;
+  }
+};
 
 // ------------------------------------------------------------------ epilogue stores
 template <int NV>
@@ -428,16 +452,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         const int pa_mn = q.a_mn, pb_mn = q.b_mn;
         const int nmain = it.kb1 - it.kb0;
         const int nkb = nmain + it.next;
+        KCursor cur(q, it.kb0, nmain);
         for (int i0 = 0; i0 < nkb; i0 += kKps) {
           const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
           if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 100)) { ok = false; break; }
           mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(cnt * kSub));
           for (int j = 0; j < cnt; ++j) {
             const int i = i0 + j;
-            const bool ext = i >= nmain;
-            const int kel = ext ? (i - nmain) * BK : (it.kb0 + i) * BK;
-            const CUtensorMap *ma = ext ? &q.tmAe : &q.tmA;
-            const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
+            const CUtensorMap *ma, *mb;
+            int kel;
+            cur.take(ma, mb, kel);
             const uint32_t sA = smem0 + stage * kStage + j * kSub, sB = sA + kStageA;
             if (!pa_mn) {
               if constexpr (BN == 16)   // decode: W0 is read exactly once; keep x, A and the split-K slabs in L2 instead
@@ -658,7 +682,7 @@ __device__ __forceinline__ Item decode_item_pair(const DevGroup &g, int item) {
   it.split = 0;
   it.kb0 = 0;
   it.kb1 = q.kb_main;
-  it.next = q.kb_ext;
+  it.next = q.kb_ext + q.kb_xtot;
   return it;
 }
 
@@ -723,11 +747,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         const int pa_mn = q.a_mn, pb_mn = q.b_mn;
         const int nmain = it.kb1 - it.kb0;
         const int nkb = nmain + it.next;
+        KCursor cur(q, it.kb0, nmain);
         for (int i = 0; i < nkb; ++i) {
-          const bool ext = i >= nmain;
-          const int kel = ext ? (i - nmain) * BK : (it.kb0 + i) * BK;
-          const CUtensorMap *ma = ext ? &q.tmAe : &q.tmA;
-          const CUtensorMap *mb = ext ? &q.tmBe : &q.tmB;
+          const CUtensorMap *ma, *mb;
+          int kel;
+          cur.take(ma, mb, kel);
           if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 400)) { ok = false; break; }
           const uint32_t fb = full0 + 8u * stage;   // the even CTA's barrier
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2u * (uint32_t)kStage);
@@ -1536,7 +1560,9 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     const TcProblem &p = probs[i];
     long long kb = (p.K + BK - 1) / BK;
     int s = p.splits < 1 ? 1 : p.splits;
-    return (kb + s - 1) / s + (p.Kext + BK - 1) / BK;
+    long long w = (kb + s - 1) / s + (p.Kext + BK - 1) / BK;
+    for (int e = 0; e < p.n_extra; ++e) w += (p.Kx[e] + BK - 1) / BK;
+    return w;
   };
   for (int i = 1; i < n; ++i)
     for (int j = i; j > 0 && weight(order[j]) > weight(order[j - 1]); --j) {
@@ -1579,6 +1605,19 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
       q.tmAe = q.tmA;
       q.tmBe = q.tmB;
     }
+    q.kb_xtot = 0;
+    if (p.n_extra < 0 || p.n_extra > kMaxExtra || (p.n_extra > 0 && q.splits > 1)) return TEMPLORA_ERR_INVALID_ARG;
+    for (int e = 0; e < kMaxExtra; ++e) {
+      q.kb_x[e] = 0;
+      q.tmXa[e] = q.tmA;
+      q.tmXb[e] = q.tmB;
+      if (e >= p.n_extra) continue;
+      if (!p.Ax[e] || !p.Bx[e] || p.Kx[e] <= 0 || ((p.ldax[e] | p.ldbx[e]) & 7)) return TEMPLORA_ERR_INVALID_ARG;
+      q.kb_x[e] = (p.Kx[e] + BK - 1) / BK;
+      q.kb_xtot += q.kb_x[e];
+      ok = ok && make_operand_map(&q.tmXa[e], p.Ax[e], p.M, p.Kx[e], p.ldax[e], p.a_mn, BM) &&
+           make_operand_map(&q.tmXb[e], p.Bx[e], p.N, p.Kx[e], p.ldbx[e], p.b_mn, box_b);
+    }
     if (!ok) return TEMPLORA_ERR_CUDA;
   }
   g.n_items = items;
@@ -1620,6 +1659,8 @@ templora_status_t tc_decode_cluster(const TcProblem *probs, int n, int n_tokens,
     q.item_start = items;
     q.a_mn = 0; q.b_mn = 0; q.out_f32 = 0;
     q.pad = p.role; q.pad3 = p.flag;
+    q.kb_xtot = 0;
+    for (int e = 0; e < kMaxExtra; ++e) { q.kb_x[e] = 0; q.tmXa[e] = q.tmA; q.tmXb[e] = q.tmB; }
     q.epi_mask = nullptr; q.epi_mask_pitch = 0; q.epi_scale = p.epi_scale;
     q.out = p.out; q.out_s0 = 1; q.out_s1 = p.out_s1; q.out_split = 0;
     items += q.m_tiles;

@@ -73,7 +73,14 @@ class Block:
     """One block of LoRA-augmented projections resident on a device, with optimizer state."""
 
     def __init__(self, b, seed, tag, projections, T, r, s, dtype="bf16", device="cuda", with_dX=True,
-                 shared_io=None, dropout_p=0.0):
+                 shared_io=None, dropout_p=0.0, input_groups=None):
+        """input_groups: lists of projection names that read the same input (e.g. [["q", "k", "v"],
+        ["gate", "up"]]): the members share the first member's x and dX tensors, and dX receives the sum
+        of their input gradients (templora_linear_t.input_group)."""
+        group_of = {}
+        for gi, names in enumerate(input_groups or []):
+            for nm in names:
+                group_of[nm] = (gi + 1, names[0])
         self.T, self.r, self.s, self.dtype = T, r, s, dtype
         self.names = [p[0] for p in projections]
         self.W0, self.state, self.lins, self.A_desc, self.B_desc = [], [], [], [], []
@@ -94,7 +101,8 @@ class Block:
             self.W0.append(W0)
             self.state.append(st)
             self.lins.append(b.linear_desc(W0, a, bb, s, dropout_p=dropout_p,
-                                           dropout_seed=inputs._key(seed, t, "dropout") & ((1 << 64) - 1)))
+                                           dropout_seed=inputs._key(seed, t, "dropout") & ((1 << 64) - 1),
+                                           input_group=group_of.get(name, (0, None))[0]))
             self.A_desc.append(b.param_desc(st["A"]["master"], st["A"]["m"], st["A"]["v"], st["A"]["grad"], st["A"]["work"]))
             self.B_desc.append(b.param_desc(st["B"]["master"], st["B"]["m"], st["B"]["v"], st["B"]["grad"], st["B"]["work"]))
             if shared_io is not None:
@@ -104,6 +112,8 @@ class Block:
                           dY=inputs.make_tensor(seed, t, "dY", (T, d_out), "normal", 1.0, dtype, device))
                 io["y"] = torch.empty((T, d_out), dtype=td, device=device)
                 io["dX"] = torch.empty((T, d_in), dtype=td, device=device) if with_dX else None
+                if name in group_of and group_of[name][1] != name:   # reads (and differentiates into) the leader's
+                    io["x"], io["dX"] = self.io[group_of[name][1]]["x"], self.io[group_of[name][1]]["dX"]
             self.io[name] = io
             self.x.append(io["x"]); self.dY.append(io["dY"]); self.y.append(io["y"]); self.dX.append(io["dX"])
         self.args = b.UpdateBlockArgs(self.lins, self.A_desc, self.B_desc, self.x, self.dY, self.y,

@@ -476,3 +476,32 @@ def test_update_block_warmup_equals_steps_composed_by_hand():
             cur.update({n: out[0][n] for n in ("A_master", "B_master", "mA", "vA", "mB", "vB")})
     for n in ("A_master", "B_master", "mA", "vA", "mB", "vB"):
         assert np.allclose(ref[0][n], cur[n], rtol=1e-13, atol=1e-15), n
+
+
+# ------------------------------------------------------------------ shared-input projections
+def test_summed_input_gradient_matches_finite_differences():
+    # q, k, v read the same x: with L = sum_i <dY_i, y_i(x)>, dL/dx is the sum of the three input
+    # gradients; L is linear in x, so central differences are exact up to rounding
+    rng = np.random.default_rng(11)
+    T, d_in, r = 4, 6, 2
+    x = rng.normal(size=(T, d_in))
+    projs = []
+    for i, d_out in enumerate((5, 3, 4)):
+        projs.append(dict(x=x, dY=rng.normal(size=(T, d_out)), W0=rng.normal(size=(d_out, d_in)), s=0.7 + i,
+                          A_master=rng.normal(size=(r, d_in)), B_master=rng.normal(size=(d_out, r)),
+                          dX_to=None if i == 0 else 0))
+    st, _ = orc.update_block(projs, 1, 0.0, 0.9, 0.999, 1e-8, 0.0)
+    assert st[1]["dX"] is st[0]["dX"] and st[2]["dX"] is st[0]["dX"]
+
+    def loss(xx):
+        return sum(np.sum(p["dY"] * orc.linear_fwd(xx, p["W0"], p["A_master"], p["B_master"], p["s"])[0]) for p in projs)
+    h = 1e-3
+    fd = np.zeros_like(x)
+    for t in range(T):
+        for k in range(d_in):
+            e = np.zeros_like(x); e[t, k] = h
+            fd[t, k] = (loss(x + e) - loss(x - e)) / (2 * h)
+    assert np.allclose(st[0]["dX"], fd, rtol=1e-9, atol=1e-9)
+    # and it is not any single projection's gradient
+    alone, _ = orc.update_block([dict(projs[0], dX_to=None)], 1, 0.0, 0.9, 0.999, 1e-8, 0.0)
+    assert not np.allclose(alone[0]["dX"], fd)

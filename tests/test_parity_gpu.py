@@ -405,3 +405,76 @@ def test_decode_repeated_calls_share_a_workspace(b):
             _decode_case(b, 23 + rep, f"dec-rep-{rep}", (1, 16, 4, 7, 2, 16)[rep], d_in, d_out, r, ws=ws)
         finally:
             b.templora_set_kernel_path(0)
+
+
+# ------------------------------------------------------------------ projections that share their input
+def _shared_input_case(b, dtype, d_in, d_outs, T, r, seed, dropout_p=0.0, epochs=1):
+    """q, k, v style: one x, one dX buffer for all projections; dX must be the sum of the input gradients."""
+    hp = hp32(dict(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0))
+    hosts = [inputs.make_linear(seed, f"sh{i}", T, d_in, do, r, dtype=dtype) for i, do in enumerate(d_outs)]
+    x_host = hosts[0]["x"]
+    x_dev = x_host.cuda()
+    devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
+    states = [make_state(h, dtype) for h in hosts]
+    dX = torch.full_like(x_dev, float("nan"))
+    lins, As, Bs, ys = [], [], [], []
+    for i, (d, st) in enumerate(zip(devs, states)):
+        a = st["A"]["work"] if dtype == "bf16" else st["A"]["master"]
+        bb = st["B"]["work"] if dtype == "bf16" else st["B"]["master"]
+        lins.append(b.linear_desc(d["W0"], a, bb, 2.0, dropout_p=dropout_p, dropout_seed=1000 + i, input_group=7))
+        As.append(b.param_desc(st["A"]["master"], st["A"]["m"], st["A"]["v"], st["A"]["grad"], st["A"]["work"]))
+        Bs.append(b.param_desc(st["B"]["master"], st["B"]["m"], st["B"]["v"], st["B"]["grad"], st["B"]["work"]))
+        ys.append(torch.full_like(d["dY"], float("nan")))
+    ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(lins, T))
+    n = len(hosts)
+    args = b.UpdateBlockArgs(lins, As, Bs, [x_dev] * n, [d["dY"] for d in devs], ys, [dX] * n)
+    step = b.templora_update_block(args, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], 0, ws)
+    assert b.templora_read_device_status(ws)[0] == 0 and step == epochs
+    projs = [dict(x=f64(x_host), dY=f64(h["dY"]), W0=f64(h["W0"]), s=2.0, A_master=f64(h["A"]), B_master=f64(h["B"]),
+                  dX_to=None if i == 0 else 0, dropout_seed=1000 + i) for i, h in enumerate(hosts)]
+    ref, _ = orc.update_block(projs, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
+                              bf16_work=(dtype == "bf16"), dropout_p=dropout_p)
+    tol = TOL[dtype]
+    assert_close("summed dX", f64(dX), ref[0]["dX"], tol)
+    for i, (q, st) in enumerate(zip(ref, states)):
+        assert_close(f"y{i}", f64(ys[i]), q["y"], tol)
+        assert_close(f"dA{i}", f64(st["A"]["grad"]), q["dA"], tol)
+        assert_close(f"dB{i}", f64(st["B"]["grad"]), q["dB"], tol)
+
+
+@pytest.mark.parametrize("d_outs", [(384, 256, 256), (640, 640)])
+def test_shared_input_summed_dx_bf16(b, d_outs):
+    _shared_input_case(b, "bf16", 512, d_outs, 300, 64, 31)
+
+
+def test_shared_input_summed_dx_two_epochs_and_single_cta_tiles(b):
+    _shared_input_case(b, "bf16", 256, (256, 384, 128), 200, 16, 32, epochs=2)
+    b.templora_set_kernel_path(2)
+    try:
+        _shared_input_case(b, "bf16", 512, (384, 256, 256), 300, 64, 31)
+    finally:
+        b.templora_set_kernel_path(0)
+
+
+def test_shared_input_summed_dx_with_dropout(b):
+    _shared_input_case(b, "bf16", 512, (384, 256, 256), 300, 64, 33, dropout_p=0.1)
+
+
+def test_shared_input_summed_dx_fp32_and_generic(b, generic_path):
+    _shared_input_case(generic_path, "f32", 96, (80, 64, 72), 50, 8, 34)
+    _shared_input_case(generic_path, "bf16", 128, (96, 64), 70, 8, 35)
+
+
+def test_shared_dx_needs_equal_input_width(b):
+    hosts = [inputs.make_linear(36, f"bad{i}", 32, di, 64, 8, dtype="bf16") for i, di in enumerate((64, 128))]
+    devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
+    states = [make_state(h, "bf16") for h in hosts]
+    lins = [b.linear_desc(d["W0"], st["A"]["work"], st["B"]["work"], 2.0, input_group=1) for d, st in zip(devs, states)]
+    As = [b.param_desc(st["A"]["master"], st["A"]["m"], st["A"]["v"], st["A"]["grad"], st["A"]["work"]) for st in states]
+    Bs = [b.param_desc(st["B"]["master"], st["B"]["m"], st["B"]["v"], st["B"]["grad"], st["B"]["work"]) for st in states]
+    ys = [torch.empty_like(d["dY"]) for d in devs]
+    dX = torch.empty((32, 128), dtype=torch.bfloat16, device="cuda")
+    ws = b.alloc_workspace(b.templora_update_block_workspace_bytes(lins, 32))
+    args = b.UpdateBlockArgs(lins, As, Bs, [d["x"] for d in devs], [d["dY"] for d in devs], ys, [dX, dX])
+    with pytest.raises(b.TemploraError):
+        b.templora_update_block(args, 1, 1e-4, 0.9, 0.999, 1e-8, 0.0, 0, ws)

@@ -624,6 +624,7 @@ constexpr int kStageB = 128 * BK * 2;            // this CTA's half of the B til
 constexpr int kStage = kStageA + kStageB;        // 32 KB per CTA and stage
 constexpr int kSmemBytes = kStages * kStage + 1024 + 1024;
 constexpr int kTmemCols = 512;                   // two 256-column accumulators
+constexpr int kPairThreads = 224;                // producer (A), MMA, four epilogue warps, producer (B)
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -686,7 +687,7 @@ __device__ __forceinline__ Item decode_item_pair(const DevGroup &g, int item) {
   return it;
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     tc_gemm_pair_kernel(const __grid_constant__ DevGroup g) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -731,8 +732,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
   const uint32_t tmem_base = *tmem_slot;
   pdl_prologue();   // the set-up above touched no global memory and may overlap the previous kernel's tail
 
-  if (warp == 0) {
-    // ===================== TMA producer (both CTAs) =====================
+  if (warp == 0 || warp == 6) {
+    // ===================== TMA producers (both CTAs): warp 0 loads the A operand, warp 6 the B operand ==========
+    // Two threads because one thread issuing every copy of a k-block was close to the critical path.
+    const bool do_a = warp == 0;
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -754,19 +757,23 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           cur.take(ma, mb, kel);
           if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 400)) { ok = false; break; }
           const uint32_t fb = full0 + 8u * stage;   // the even CTA's barrier
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2u * (uint32_t)kStage);
+          // one announcement covers the bytes of both operands of both CTAs (bytes may land before it)
+          if (rank == 0 && do_a) mbar_arrive_expect_tx(full_bar(stage), 2u * (uint32_t)kStage);
           const uint32_t sA = smem0 + stage * kStage, sB = sA + kStageA;
-          if (!pa_mn) {
-            tma_load_2d_pair(sA, ma, fb, kel, m0);
-          } else {
+          if (do_a) {
+            if (!pa_mn) {
+              tma_load_2d_pair(sA, ma, fb, kel, m0);
+            } else {
 #pragma unroll
-            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sA + b * 8192, ma, fb, m0 + b * 64, kel);
-          }
-          if (!pb_mn) {
-            tma_load_2d_pair(sB, mb, fb, kel, n0);
+              for (int b = 0; b < 2; ++b) tma_load_2d_pair(sA + b * 8192, ma, fb, m0 + b * 64, kel);
+            }
           } else {
+            if (!pb_mn) {
+              tma_load_2d_pair(sB, mb, fb, kel, n0);
+            } else {
 #pragma unroll
-            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sB + b * 8192, mb, fb, n0 + b * 64, kel);
+              for (int b = 0; b < 2; ++b) tma_load_2d_pair(sB + b * 8192, mb, fb, n0 + b * 64, kel);
+            }
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -1425,7 +1432,7 @@ templora_status_t launch_pair(const DevGroup &g, DeviceInfo *di, cudaStream_t st
   if (g.n_items < pairs) pairs = g.n_items;
   {
     LaunchScope scope(kKindTcMain, st);
-    TL_CUDA_CHECK(launch_pdl(pair::tc_gemm_pair_kernel, dim3(2 * pairs), dim3(kThreads), pair::kSmemBytes, st, g));
+    TL_CUDA_CHECK(launch_pdl(pair::tc_gemm_pair_kernel, dim3(2 * pairs), dim3(pair::kPairThreads), pair::kSmemBytes, st, g));
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;

@@ -31,6 +31,7 @@ namespace {
 
 constexpr int BM = 128, BK = 64;
 constexpr int kThreads = 192;
+constexpr int kThreads2 = 224;   // single-CTA GEMM kernel: one more warp, the second TMA producer
 constexpr int kSched = 4;  // depth of the work-item ring between the producer and its consumers
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
@@ -374,7 +375,7 @@ __device__ __forceinline__ void masked_add_row(const DevProb &q, uint32_t t_row,
 
 // ------------------------------------------------------------------ the kernel
 template <int BN>
-__global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ DevGroup g) {
+__global__ void __launch_bounds__(kThreads2, 1) tc_gemm_kernel(const __grid_constant__ DevGroup g) {
   constexpr int kStages = Cfg<BN>::kStages;
   constexpr int kStage = Cfg<BN>::kStage;
   constexpr int kSub = Cfg<BN>::kSub;
@@ -411,7 +412,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     mbar_init(drain_bar, 1);
     for (int s = 0; s < kSched; ++s) {
       mbar_init(sfull_bar(s), 1);
-      mbar_init(sempty_bar(s), 5);  // the MMA thread + one lane of each epilogue warp
+      mbar_init(sempty_bar(s), 6);  // the B-operand producer, the MMA thread, one lane of each epilogue warp
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -430,7 +431,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
   pdl_prologue();   // the set-up above touched no global memory and may overlap the previous kernel's tail
 
   if (warp == 0) {
-    // ===================== TMA producer =====================
+    // ===================== TMA producer: hands out the items and loads the A operand =====================
+    // (the B operand is loaded by warp 6: one thread issuing every copy was close to the critical path)
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -448,8 +450,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         const int next_item = (int)gridDim.x + atomicAdd(&g.status->sched_next, 1);  // drawn early, used late
         const Item it = decode_item(g, item);
         const DevProb &q = g.p[it.p];
-        const int n0 = it.nt * BN;
-        const int pa_mn = q.a_mn, pb_mn = q.b_mn;
+        const int pa_mn = q.a_mn;
         const int nmain = it.kb1 - it.kb0;
         const int nkb = nmain + it.next;
         KCursor cur(q, it.kb0, nmain);
@@ -458,11 +459,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
           if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 100)) { ok = false; break; }
           mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(cnt * kSub));
           for (int j = 0; j < cnt; ++j) {
-            const int i = i0 + j;
             const CUtensorMap *ma, *mb;
             int kel;
             cur.take(ma, mb, kel);
-            const uint32_t sA = smem0 + stage * kStage + j * kSub, sB = sA + kStageA;
+            const uint32_t sA = smem0 + stage * kStage + j * kSub;
             if (!pa_mn) {
               if constexpr (BN == 16)   // decode: W0 is read exactly once; keep x, A and the split-K slabs in L2 instead
                 tma_load_2d_hint(sA, ma, full_bar(stage), kel, it.m0, stream_policy);
@@ -471,13 +471,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             } else {
 #pragma unroll
               for (int b = 0; b < BM / 64; ++b) tma_load_2d(sA + b * 8192, ma, full_bar(stage), it.m0 + b * 64, kel);
-            }
-            if (!pb_mn) {
-              tma_load_2d(sB, mb, full_bar(stage), kel, n0);
-            } else {
-#pragma unroll
-              for (int b = 0; b < (BN >= 64 ? BN / 64 : 1); ++b)
-                tma_load_2d(sB + b * 8192, mb, full_bar(stage), n0 + b * 64, kel);
             }
           }
           ++issued;
@@ -494,6 +487,45 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
           uint32_t ph = (uint32_t)((idx / kStages) & 1);
           const unsigned long long t0 = globaltimer_ns();
           while (!mbar_try(full_bar(s), ph) && globaltimer_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 6) {
+    // ===================== second TMA producer: the B operand =====================
+    if (lane == 0) {
+      int stage = 0, sslot = 0;
+      uint32_t phase = 0, sphase = 0;
+      bool ok = true;
+      while (ok) {
+        if (!mbar_wait(sfull_bar(sslot), sphase, abort_flag, g.status, 120)) { ok = false; break; }
+        const int item = sched_ring[sslot];
+        mbar_arrive(sempty_bar(sslot));
+        if (++sslot == kSched) { sslot = 0; sphase ^= 1u; }
+        if (item >= g.n_items) break;
+        const Item it = decode_item(g, item);
+        const DevProb &q = g.p[it.p];
+        const int n0 = it.nt * BN;
+        const int pb_mn = q.b_mn;
+        const int nmain = it.kb1 - it.kb0;
+        const int nkb = nmain + it.next;
+        KCursor cur(q, it.kb0, nmain);
+        for (int i0 = 0; i0 < nkb; i0 += kKps) {
+          const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
+          if (!mbar_wait_fast(empty_bar(stage), phase ^ 1u, abort_flag, g.status, 121)) { ok = false; break; }
+          for (int j = 0; j < cnt; ++j) {
+            const CUtensorMap *ma, *mb;
+            int kel;
+            cur.take(ma, mb, kel);
+            const uint32_t sB = smem0 + stage * kStage + j * kSub + kStageA;
+            if (!pb_mn) {
+              tma_load_2d(sB, mb, full_bar(stage), kel, n0);
+            } else {
+#pragma unroll
+              for (int b = 0; b < (BN >= 64 ? BN / 64 : 1); ++b)
+                tma_load_2d(sB + b * 8192, mb, full_bar(stage), n0 + b * 64, kel);
+            }
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -1415,7 +1447,7 @@ templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream
   {
     LaunchScope scope(g.p[0].epi_mask ? kKindTcDropoutTerm
                                        : (BN == 256 ? kKindTcMain : (BN == 64 ? kKindTcSkinny : kKindTcDecode)), st);
-    TL_CUDA_CHECK(launch_pdl(tc_gemm_kernel<BN>, dim3(grid), dim3(kThreads), Cfg<BN>::kSmemBytes, st, g));
+    TL_CUDA_CHECK(launch_pdl(tc_gemm_kernel<BN>, dim3(grid), dim3(kThreads2), Cfg<BN>::kSmemBytes, st, g));
   }
   TL_CUDA_CHECK(cudaGetLastError());
   return TEMPLORA_OK;

@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the dominant kernel (bytes), from an ncu capture summarised under
 # profiles/; valid only while the kernel source is the one that was profiled.
 SHARED_INPUTS = [["q", "k", "v"], ["gate", "up"]]   # projections of a decoder block that read the same tensor
-TRAFFIC = {"tc_gemm_sha1": "2adce7a4be89190307bd16910780a2efe7dbf3bf", "bytes_per_launch": 1356845608}
+TRAFFIC = {"tc_gemm_sha1": "b8a8aeb20883793ca0e0004e21d070f2e9fc3b4e", "bytes_per_launch": 1284111488}
 
 
 def load_peaks():

@@ -700,59 +700,69 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
   }
   TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
   TL_TRY(reduce_partials_batch(jobs, nj, st));
-  np = 0;
-  // Projections given the same dX buffer (they share their input) get ONE problem: the products of the
-  // later ones are appended to the first one's k-loop, so the sum forms in the accumulator.
-  int owner[kGroup], rank_in_set[kGroup], prob_of[kGroup], max_rank = 0;
-  for (int i = 0; i < n; ++i) {
-    owner[i] = i; rank_in_set[i] = 0; prob_of[i] = -1;
-    if (!(dX && dX[i])) continue;
-    for (int k = 0; k < i && proj[i].input_group != 0; ++k)
-      if (dX[k] && proj[k].input_group == proj[i].input_group) { owner[i] = owner[k]; ++rank_in_set[i]; }
-    if (rank_in_set[i] > max_rank) max_rank = rank_in_set[i];
-  }
-  for (int i = 0; i < n; ++i) {
-    probs[np++] = prob_y(proj + i, T, x[i], b.Us[i], y[i]);
-    if (!(dX && dX[i])) continue;
-    if (owner[i] == i) {
-      prob_of[i] = np;
-      probs[np] = prob_dX(proj + i, T, dY[i], b.Vs[i], dX[i]);
-      if (b.drop[i].xd) probs[np].Kext = 0;   // masked rank-r term: second pass below
-      ++np;
-    } else {
-      TcProblem &o = probs[prob_of[owner[i]]];
-      if (proj[i].d_in != proj[owner[i]].d_in || o.n_extra + 2 > 4) return TEMPLORA_ERR_INVALID_ARG;
-      int e = o.n_extra;
-      o.Ax[e] = dY[i]; o.ldax[e] = proj[i].d_out; o.Bx[e] = proj[i].W0; o.ldbx[e] = proj[i].d_in; o.Kx[e] = proj[i].d_out;
-      ++e;
-      if (!b.drop[i].xd) {
-        o.Ax[e] = b.Vs[i]; o.ldax[e] = proj[i].r; o.Bx[e] = proj[i].A; o.ldbx[e] = proj[i].d_in; o.Kx[e] = proj[i].r;
-        ++e;
-      }
-      o.n_extra = e;
+  // dB and dA go before the frozen-weight GEMMs: they re-read x and dY, which the U, V launch has just
+  // pulled through L2 (the big GEMMs stream 1.1 GB and would flush them)
+  auto launch_grads = [&]() -> templora_status_t {
+    np = 0; nj = 0;
+    for (int i = 0; i < n; ++i) {
+      const templora_linear_t *l = proj + i;
+      float *gB = const_cast<float *>(Bs[i].grad), *gA = const_cast<float *>(As[i].grad);
+      probs[np++] = prob_dB(l, T, dY[i], b.Us[i], b.sb[i] > 1 ? b.dBpart[i] : gB, b.sb[i]);
+      probs[np++] = prob_dA(l, T, xb[i], b.Vs[i], b.sa[i] > 1 ? b.dApart[i] : gA, b.sa[i]);
+      const long long nb = (long long)l->d_out * l->r, na = (long long)l->d_in * l->r;
+      if (b.sb[i] > 1) jobs[nj++] = ReduceJob{b.dBpart[i], b.sb[i], nb, nb, 1.f, 1.f, gB, 0, nullptr};
+      if (b.sa[i] > 1) jobs[nj++] = ReduceJob{b.dApart[i], b.sa[i], na, na, 1.f, 1.f, gA, 0, nullptr};
     }
-  }
-  TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, use_pairs()));
-  // masked rank-r terms: read-modify-write passes; those aimed at the same buffer go in successive launches
-  for (int round = 0; round <= max_rank; ++round) {
+    TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
+    if (nj) TL_TRY(reduce_partials_batch(jobs, nj, st));
+    return TEMPLORA_OK;
+  };
+  auto launch_main = [&]() -> templora_status_t {
     np = 0;
-    for (int i = 0; i < n; ++i)
-      if (dX && dX[i] && b.drop[i].xd && rank_in_set[i] == round)
-        probs[np++] = prob_dX_dropout_term(proj + i, T, b.Vs[i], dX[i], b.drop[i]);
-    if (np) TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, 0));
-  }
-  np = 0; nj = 0;
-  for (int i = 0; i < n; ++i) {
-    const templora_linear_t *l = proj + i;
-    float *gB = const_cast<float *>(Bs[i].grad), *gA = const_cast<float *>(As[i].grad);
-    probs[np++] = prob_dB(l, T, dY[i], b.Us[i], b.sb[i] > 1 ? b.dBpart[i] : gB, b.sb[i]);
-    probs[np++] = prob_dA(l, T, xb[i], b.Vs[i], b.sa[i] > 1 ? b.dApart[i] : gA, b.sa[i]);
-    const long long nb = (long long)l->d_out * l->r, na = (long long)l->d_in * l->r;
-    if (b.sb[i] > 1) jobs[nj++] = ReduceJob{b.dBpart[i], b.sb[i], nb, nb, 1.f, 1.f, gB, 0, nullptr};
-    if (b.sa[i] > 1) jobs[nj++] = ReduceJob{b.dApart[i], b.sa[i], na, na, 1.f, 1.f, gA, 0, nullptr};
-  }
-  TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
-  if (nj) TL_TRY(reduce_partials_batch(jobs, nj, st));
+    // Projections given the same dX buffer (they share their input) get ONE problem: the products of the
+    // later ones are appended to the first one's k-loop, so the sum forms in the accumulator.
+    int owner[kGroup], rank_in_set[kGroup], prob_of[kGroup], max_rank = 0;
+    for (int i = 0; i < n; ++i) {
+      owner[i] = i; rank_in_set[i] = 0; prob_of[i] = -1;
+      if (!(dX && dX[i])) continue;
+      for (int k = 0; k < i && proj[i].input_group != 0; ++k)
+        if (dX[k] && proj[k].input_group == proj[i].input_group) { owner[i] = owner[k]; ++rank_in_set[i]; }
+      if (rank_in_set[i] > max_rank) max_rank = rank_in_set[i];
+    }
+    for (int i = 0; i < n; ++i) {
+      probs[np++] = prob_y(proj + i, T, x[i], b.Us[i], y[i]);
+      if (!(dX && dX[i])) continue;
+      if (owner[i] == i) {
+        prob_of[i] = np;
+        probs[np] = prob_dX(proj + i, T, dY[i], b.Vs[i], dX[i]);
+        if (b.drop[i].xd) probs[np].Kext = 0;   // masked rank-r term: second pass below
+        ++np;
+      } else {
+        TcProblem &o = probs[prob_of[owner[i]]];
+        if (proj[i].d_in != proj[owner[i]].d_in || o.n_extra + 2 > 4) return TEMPLORA_ERR_INVALID_ARG;
+        int e = o.n_extra;
+        o.Ax[e] = dY[i]; o.ldax[e] = proj[i].d_out; o.Bx[e] = proj[i].W0; o.ldbx[e] = proj[i].d_in; o.Kx[e] = proj[i].d_out;
+        ++e;
+        if (!b.drop[i].xd) {
+          o.Ax[e] = b.Vs[i]; o.ldax[e] = proj[i].r; o.Bx[e] = proj[i].A; o.ldbx[e] = proj[i].d_in; o.Kx[e] = proj[i].r;
+          ++e;
+        }
+        o.n_extra = e;
+      }
+    }
+    TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, use_pairs()));
+    // masked rank-r terms: read-modify-write passes; those aimed at the same buffer go in successive launches
+    for (int round = 0; round <= max_rank; ++round) {
+      np = 0;
+      for (int i = 0; i < n; ++i)
+        if (dX && dX[i] && b.drop[i].xd && rank_in_set[i] == round)
+          probs[np++] = prob_dX_dropout_term(proj + i, T, b.Vs[i], dX[i], b.drop[i]);
+      if (np) TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, 0));
+    }
+    return TEMPLORA_OK;
+  };
+  TL_TRY(launch_grads());
+  TL_TRY(launch_main());
   return TEMPLORA_OK;
 }
 

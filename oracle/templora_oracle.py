@@ -246,3 +246,38 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
         if p.get("dX_to") is not None:
             q["dX"] = st[p["dX_to"]]["dX"]
     return st, step
+
+
+# ---------------------------------------------------------------------------
+# The steps on either side of the projections inside a decoder block's update
+# ("Train Theta_k" runs a whole Llama-style block: RMSNorm -> q,k,v ... and
+# gate, up -> SiLU(gate) * up -> down).  Plain definitions, fp64.
+# ---------------------------------------------------------------------------
+def swiglu_fwd(gate, up):
+    """h = SiLU(gate) * up with SiLU(g) = g * sigmoid(g) (the Llama MLP's gating)."""
+    g, u = _f64(gate), _f64(up)
+    return g / (1.0 + np.exp(-g)) * u
+
+
+def swiglu_bwd(gate, up, dh):
+    """Gradients of h = SiLU(gate) * up:  dgate = dh * up * SiLU'(gate),  dup = dh * SiLU(gate),
+    with SiLU'(g) = sigmoid(g) * (1 + g * (1 - sigmoid(g)))."""
+    g, u, d = _f64(gate), _f64(up), _f64(dh)
+    sg = 1.0 / (1.0 + np.exp(-g))
+    return d * u * sg * (1.0 + g * (1.0 - sg)), d * g * sg
+
+
+def rmsnorm_fwd(x, w, eps):
+    """y[t, j] = x[t, j] / sqrt(mean_j x[t, j]^2 + eps) * w[j]  (Llama's RMSNorm; w is frozen here)."""
+    x, w = _f64(x), _f64(w)
+    rstd = 1.0 / np.sqrt(np.mean(x * x, axis=1, keepdims=True) + eps)
+    return x * rstd * w
+
+
+def rmsnorm_bwd(x, w, dy, eps):
+    """dx of y = rmsnorm(x):  with xh = x * rstd and g = w * dy,
+    dx = rstd * (g - xh * mean_j(xh * g)).  No weight gradient: the norm weights are not trained."""
+    x, w, dy = _f64(x), _f64(w), _f64(dy)
+    rstd = 1.0 / np.sqrt(np.mean(x * x, axis=1, keepdims=True) + eps)
+    xh, g = x * rstd, w * dy
+    return rstd * (g - xh * np.mean(xh * g, axis=1, keepdims=True))

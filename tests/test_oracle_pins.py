@@ -505,3 +505,48 @@ def test_summed_input_gradient_matches_finite_differences():
     # and it is not any single projection's gradient
     alone, _ = orc.update_block([dict(projs[0], dX_to=None)], 1, 0.0, 0.9, 0.999, 1e-8, 0.0)
     assert not np.allclose(alone[0]["dX"], fd)
+
+
+# ------------------------------------------------------------------ SiLU gating and RMSNorm
+def _fd(f, x, h=1e-6):
+    g = np.zeros_like(x)
+    it = np.nditer(x, flags=["multi_index"])
+    for _ in it:
+        e = np.zeros_like(x); e[it.multi_index] = h
+        g[it.multi_index] = (f(x + e) - f(x - e)) / (2 * h)
+    return g
+
+
+def test_swiglu_values_and_gradients():
+    # SiLU(0) = 0, SiLU'(0) = 1/2, SiLU(g) -> g for large g, -> 0 for very negative g
+    assert orc.swiglu_fwd(np.array([[0.0]]), np.array([[3.0]]))[0, 0] == 0.0
+    dg, du = orc.swiglu_bwd(np.array([[0.0]]), np.array([[3.0]]), np.array([[2.0]]))
+    assert dg[0, 0] == pytest.approx(2.0 * 3.0 * 0.5, rel=1e-15) and du[0, 0] == 0.0
+    assert orc.swiglu_fwd(np.array([[40.0]]), np.array([[1.0]]))[0, 0] == pytest.approx(40.0, rel=1e-15)
+    assert abs(orc.swiglu_fwd(np.array([[-40.0]]), np.array([[1.0]]))[0, 0]) < 1e-15
+    # textbook value: SiLU(1) = 1 / (1 + e^-1)
+    assert orc.swiglu_fwd(np.array([[1.0]]), np.array([[1.0]]))[0, 0] == pytest.approx(0.7310585786300049, rel=1e-15)
+    rng = np.random.default_rng(3)
+    g, u, dh = rng.normal(size=(3, 4)), rng.normal(size=(3, 4)), rng.normal(size=(3, 4))
+    dg, du = orc.swiglu_bwd(g, u, dh)
+    assert np.allclose(dg, _fd(lambda z: np.sum(dh * orc.swiglu_fwd(z, u)), g), rtol=1e-7, atol=1e-9)
+    assert np.allclose(du, _fd(lambda z: np.sum(dh * orc.swiglu_fwd(g, z)), u), rtol=1e-7, atol=1e-9)
+
+
+def test_rmsnorm_values_and_gradients():
+    # a row of equal entries c normalises to sign(c) * w (eps = 0); scaling a row leaves y unchanged
+    w = np.array([1.0, 2.0, -3.0, 0.5])
+    assert np.allclose(orc.rmsnorm_fwd(np.full((1, 4), -2.5), w, 0.0), -w, rtol=1e-15)
+    rng = np.random.default_rng(4)
+    x, dy = rng.normal(size=(3, 4)), rng.normal(size=(3, 4))
+    assert np.allclose(orc.rmsnorm_fwd(7.0 * x, w, 0.0), orc.rmsnorm_fwd(x, w, 0.0), rtol=1e-13)
+    # hand value: x = (3, 4), w = 1: rms = sqrt(12.5)
+    assert np.allclose(orc.rmsnorm_fwd(np.array([[3.0, 4.0]]), np.ones(2), 0.0), np.array([[3.0, 4.0]]) / np.sqrt(12.5))
+    # eps enters under the root
+    assert orc.rmsnorm_fwd(np.array([[0.0, 0.0]]), np.ones(2), 1e-6)[0, 0] == 0.0
+    assert orc.rmsnorm_fwd(np.array([[1.0, 1.0]]), np.ones(2), 3.0)[0, 0] == pytest.approx(0.5, rel=1e-15)
+    for eps in (0.0, 1e-5, 0.3):
+        dx = orc.rmsnorm_bwd(x, w, dy, eps)
+        assert np.allclose(dx, _fd(lambda z: np.sum(dy * orc.rmsnorm_fwd(z, w, eps)), x), rtol=1e-6, atol=1e-8)
+    # scale invariance of y (eps = 0) makes dx orthogonal to x, row by row
+    assert np.allclose(np.sum(orc.rmsnorm_bwd(x, w, dy, 0.0) * x, axis=1), 0.0, atol=1e-13)

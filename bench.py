@@ -327,6 +327,11 @@ def run_ours(args):
     if not args.no_decode:
         decode = decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=args.decode_blocks)
 
+    # ---- SiLU gating and RMSNorm (the element-wise steps of a block update beside the projections) ----
+    block_ops = None
+    if not args.no_decode:
+        block_ops = block_ops_bandwidth(b, torch, inputs, dev, peaks)
+
     # ---- parallelized deployment: the update on one stream, decode on another, SMs split ----
     parallel = None
     if not args.no_parallel and default_workload and stacked <= 1:
@@ -348,7 +353,8 @@ def run_ours(args):
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": n_e2e, "what": "per step: x and dY of the 7 projections from pinned host memory in (double-buffered, copy of step i+1 overlaps compute of step i), updated bf16 A and B out"},
                 "gpu_launches": int(launches), "roofline": roofline, "kernel_time_share": kernel_share,
-                "clocks": clk.summary(), "cpu_baseline": cpu, "decode": decode, "parallel_deployment": parallel}
+                "clocks": clk.summary(), "cpu_baseline": cpu, "decode": decode, "block_ops": block_ops,
+                "parallel_deployment": parallel}
         print(json.dumps(line))
     ranks.close()
     return 0
@@ -402,6 +408,42 @@ def parallel_deployment(b, torch, runtime, blk, hp, update_sms=116, decode_sms=3
                         "same block on another; 'alone' figures keep the SM caps"}
     finally:
         dep.close()
+
+
+def block_ops_bandwidth(b, torch, inputs, dev, peaks, T=4096, reps=20):
+    """HBM throughput of the SiLU-gating and RMSNorm kernels at 7B widths (bf16; T rows of 11008 for the
+    gating, 4 T rows of 4096 for the norm so that a launch outlasts the host's call overhead; four buffer
+    sets in rotation so that each launch's tensors come from DRAM).  Bytes = every tensor read or written once."""
+    Tn = 4 * T
+    n_rot = 4
+    mk = lambda tag, shape: inputs.make_tensor(0, "blockops", tag, shape, "normal", 1.0, "bf16", dev)
+    sets = [dict(g=mk(f"g{i}", (T, 11008)), u=mk(f"u{i}", (T, 11008)), dh=mk(f"dh{i}", (T, 11008)),
+                 o0=torch.empty((T, 11008), dtype=torch.bfloat16, device=dev),
+                 o1=torch.empty((T, 11008), dtype=torch.bfloat16, device=dev),
+                 x=mk(f"x{i}", (Tn, 4096)), dy=mk(f"dy{i}", (Tn, 4096)),
+                 y=torch.empty((Tn, 4096), dtype=torch.bfloat16, device=dev)) for i in range(n_rot)]
+    w = inputs.make_tensor(0, "blockops", "w", (4096,), "uniform", 1.0, "bf16", dev)
+    ops = {
+        "swiglu_fwd": (lambda s: b.templora_swiglu_fwd(s["g"], s["u"], s["o0"]), 3 * T * 11008 * 2),
+        "swiglu_bwd": (lambda s: b.templora_swiglu_bwd(s["g"], s["u"], s["dh"], s["o0"], s["o1"]), 5 * T * 11008 * 2),
+        "rmsnorm_fwd": (lambda s: b.templora_rmsnorm_fwd(s["x"], w, 1e-5, s["y"]), 2 * Tn * 4096 * 2),
+        "rmsnorm_bwd": (lambda s: b.templora_rmsnorm_bwd(s["x"], w, s["dy"], 1e-5, s["y"]), 3 * Tn * 4096 * 2),
+    }
+    out = {"rows_gating": T, "rows_norm": Tn, "dtype": "bf16"}
+    for name, (fn, nbytes) in ops.items():
+        for s in sets:
+            fn(s)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for s in sets:
+                fn(s)
+        e1.record()
+        torch.cuda.synchronize()
+        sec = e0.elapsed_time(e1) / 1e3 / (reps * n_rot)
+        out[name] = {"us": sec * 1e6, "GBps": nbytes / sec / 1e9, "frac_of_measured_hbm": nbytes / sec / 1e9 / peaks["hbm"]}
+    return out
 
 
 def decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=32, reps=5):

@@ -225,6 +225,32 @@ const char *templora_status_string(templora_status_t st);
 templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *code, int32_t *where);
 
 /*
+ * The element-wise steps on either side of the projections when "Train Theta_k" (Algorithm 1) runs over
+ * a Llama-style decoder block: the MLP's gating between gate/up and down, and the RMSNorm in front of
+ * q,k,v and of gate,up.  The paper names neither (it trains stock Llama-2 / Yi blocks); the formulas are
+ * those models' definitions.  All tensors are contiguous DEVICE buffers of `dtype` (templora_dtype_t),
+ * 16-byte aligned; arithmetic in fp32; nothing is allocated; errors as for the other entry points.
+ *
+ * SiLU gating over n elements (any shape, flattened):
+ *   fwd:  h = SiLU(gate) * up,            SiLU(g) = g * sigmoid(g)
+ *   bwd:  dgate = dh * up * SiLU'(gate),  dup = dh * SiLU(gate),  SiLU'(g) = sigmoid(g) (1 + g (1 - sigmoid(g)))
+ */
+templora_status_t templora_swiglu_fwd(int64_t n, int32_t dtype, const void *gate, const void *up, void *h, void *stream);
+templora_status_t templora_swiglu_bwd(int64_t n, int32_t dtype, const void *gate, const void *up, const void *dh,
+                                      void *dgate, void *dup, void *stream);
+
+/*
+ * RMSNorm over the rows of x [T, d] with weight w [d] (frozen: no weight gradient):
+ *   fwd:  y[t, j]  = x[t, j] * rstd[t] * w[j],   rstd[t] = 1 / sqrt(mean_j x[t, j]^2 + eps)
+ *   bwd:  dx[t, j] = rstd[t] * (w[j] dy[t, j] - xh[t, j] * mean_j(xh[t, j] w[j] dy[t, j])),  xh = x * rstd
+ * The backward recomputes rstd from x.
+ */
+templora_status_t templora_rmsnorm_fwd(int32_t T, int32_t d, int32_t dtype, const void *x, const void *w, float eps,
+                                       void *y, void *stream);
+templora_status_t templora_rmsnorm_bwd(int32_t T, int32_t d, int32_t dtype, const void *x, const void *w, const void *dy,
+                                       float eps, void *dx, void *stream);
+
+/*
  * Failure-detection self-test (the paper has no counterpart).  Enqueues one tiny kernel that
  * waits, the way the GEMM kernels wait for their copies, on a barrier that nothing signals.
  * After limit_ms (1..1000) it records TEMPLORA_ERR_TIMEOUT in the status record at the head of
@@ -286,7 +312,8 @@ templora_status_t templora_decode_fwd_noalloc(const templora_linear_t *lin, int3
  * every launch (which costs the timed kernel and its successor their early scheduling).  Kernel classes: 0 tensor-core GEMM
  * with 256-wide tiles (y, dX), 1 tensor-core GEMM with 64-wide tiles (U, V, dA, dB),
  * 2 tensor-core GEMM with 16-wide tiles (decode), 3 partial reduction, 4 AdamW,
- * 5 generic GEMM, 6 decode finish, 7 dropout mask, 8 masked rank-r pass of dX.  Process-wide.
+ * 5 generic GEMM, 6 decode finish, 7 dropout mask, 8 masked rank-r pass of dX, 9 SiLU gating and
+ * RMSNorm.  Process-wide.
  */
 void templora_timing_enable(int32_t kind_mask);
 

@@ -23,12 +23,13 @@ EXPORTS = [
     "templora_timing_enable", "templora_timing_read", "templora_decode_fwd_noalloc",
     "templora_decode_block_workspace_bytes", "templora_decode_block_fwd", "templora_update_block_batched",
     "templora_set_stream_sm_limit", "templora_selftest_bounded_wait", "templora_lr_at_step",
-    "templora_update_block_warmup",
+    "templora_update_block_warmup", "templora_swiglu_fwd", "templora_swiglu_bwd", "templora_rmsnorm_fwd",
+    "templora_rmsnorm_bwd",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 (KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
- KIND_TC_DROPOUT_TERM) = range(9)
-N_KINDS = 9
+ KIND_TC_DROPOUT_TERM, KIND_BLOCK_OPS) = range(10)
+N_KINDS = 10
 
 
 class LinearDesc(C.Structure):
@@ -77,6 +78,14 @@ def _load():
     lib.templora_update_block_warmup.restype = i32
     lib.templora_update_block_warmup.argtypes = [LP, PP, PP, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                                  C.POINTER(vp), i32, f32, i64, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_swiglu_fwd.restype = i32
+    lib.templora_swiglu_fwd.argtypes = [i64, i32, vp, vp, vp, vp]
+    lib.templora_swiglu_bwd.restype = i32
+    lib.templora_swiglu_bwd.argtypes = [i64, i32, vp, vp, vp, vp, vp, vp]
+    lib.templora_rmsnorm_fwd.restype = i32
+    lib.templora_rmsnorm_fwd.argtypes = [i32, i32, i32, vp, vp, f32, vp, vp]
+    lib.templora_rmsnorm_bwd.restype = i32
+    lib.templora_rmsnorm_bwd.argtypes = [i32, i32, i32, vp, vp, vp, f32, vp, vp]
     lib.templora_lr_at_step.restype = f32
     lib.templora_lr_at_step.argtypes = [f32, i64, i64]
     lib.templora_selftest_bounded_wait.restype = i32
@@ -239,6 +248,28 @@ def templora_update_block_warmup(args, batch_tokens, epochs, lr, warmup_steps, b
                                             eps, weight_decay, C.byref(st), _ptr(ws), ws.numel(), _stream(stream)),
            "templora_update_block_warmup")
     return st.value
+
+
+def templora_swiglu_fwd(gate, up, h, stream=None):
+    """h = SiLU(gate) * up, element-wise over contiguous tensors of one shape and dtype."""
+    _check(lib.templora_swiglu_fwd(gate.numel(), dtype_code(gate), _ptr(gate), _ptr(up), _ptr(h), _stream(stream)),
+           "templora_swiglu_fwd")
+
+
+def templora_swiglu_bwd(gate, up, dh, dgate, dup, stream=None):
+    _check(lib.templora_swiglu_bwd(gate.numel(), dtype_code(gate), _ptr(gate), _ptr(up), _ptr(dh), _ptr(dgate), _ptr(dup),
+                                   _stream(stream)), "templora_swiglu_bwd")
+
+
+def templora_rmsnorm_fwd(x, w, eps, y, stream=None):
+    """y = x / sqrt(mean(x^2) + eps) * w over the rows of a contiguous [T, d] tensor."""
+    _check(lib.templora_rmsnorm_fwd(x.shape[0], x.shape[1], dtype_code(x), _ptr(x), _ptr(w), eps, _ptr(y),
+                                    _stream(stream)), "templora_rmsnorm_fwd")
+
+
+def templora_rmsnorm_bwd(x, w, dy, eps, dx, stream=None):
+    _check(lib.templora_rmsnorm_bwd(x.shape[0], x.shape[1], dtype_code(x), _ptr(x), _ptr(w), _ptr(dy), eps, _ptr(dx),
+                                    _stream(stream)), "templora_rmsnorm_bwd")
 
 
 def templora_lr_at_step(lr, step, warmup_steps):

@@ -49,7 +49,8 @@ enum KernelKind {
   kKindDecodeFinish = 6,
   kKindDropout = 7,        // dropout mask + masked copy of x
   kKindTcDropoutTerm = 8,  // tensor-core second pass adding the masked rank-r term to dX
-  kKindCount = 9
+  kKindBlockOps = 9,       // SiLU gating and RMSNorm, forward and backward
+  kKindCount = 10
 };
 // Construct right before a kernel launch and destroy right after it.
 class LaunchScope {

@@ -642,13 +642,47 @@ __global__ void __launch_bounds__(kThreads2, 1) tc_gemm_kernel(const __grid_cons
   }
 }
 
+// ------------------------------------------------------------------ helpers shared by the cluster kernels
+__device__ __forceinline__ void st_cluster_s32(uint32_t addr, int v) {
+  asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+// Arrive on a peer's barrier to say "I have finished reading" (nothing of mine needs to become visible).
+__device__ __forceinline__ void mbar_arrive_remote_plain(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_acq_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait whose success also makes a peer's earlier shared-memory stores (released at cluster scope) visible.
+__device__ __noinline__ bool mbar_wait_acq_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                   DeviceStatus *st, int where) {
+  for (int i = 0; i < 4096; ++i)
+    if (mbar_try_acq_cluster(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  while (true) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_acq_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      if (st && atomicCAS(&st->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) st->where = where;
+      __threadfence();
+      return false;
+    }
+  }
+}
+
 // ------------------------------------------------------------------ CTA-pair kernel (256 x 256 tiles)
 // Two CTAs of a cluster (one TPC) share one 256 x 256 output tile: each loads its own 128 rows of
 // the A operand and its own 128-column half of the B operand, and the even CTA issues
 // tcgen05.mma.cta_group::2 (M = 256), which reads both halves of B from the two CTAs' shared
 // memory.  Per flop this moves 1.5x fewer operand bytes from L2 into shared memory than 128 x 256
 // tiles on single CTAs, which is what bounds the frozen-weight GEMMs.  Each CTA drains its own
-// 128 x 256 half of the accumulator from its own TMEM.  Items are dealt round-robin to the pairs.
+// 128 x 256 half of the accumulator from its own TMEM.  Items are handed out dynamically, heaviest first.
 namespace pair {
 
 constexpr int kStages = 6;
@@ -732,6 +766,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
   const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
   volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + kStages * kStage + 512);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 516);
+  // Work items are handed out dynamically: the even CTA's A-operand producer draws them from the counter in
+  // the workspace head (heaviest problems come first, so this is longest-processing-time-first scheduling)
+  // and writes each into the item rings of both CTAs; every other role takes its items from its CTA's ring.
+  volatile int *sched_ring = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 528);
+  const uint32_t ring0 = bar0 + 528;
+  auto sfull_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 5 + s); };            // one per CTA
+  auto sempty_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 5 + kSched + s); };  // used in the even CTA
+  // readers of a ring slot: even CTA: B producer, MMA thread, 4 epilogue warps; odd CTA: both producers, 4 epilogue warps
+  constexpr int kRingReaders = 12;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();      // 0: issues the MMAs; 1: its peer
@@ -747,6 +790,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       mbar_init(tempty_bar(a), 8);  // four epilogue warps in each CTA
     }
     mbar_init(drain_bar, 1);
+    for (int s = 0; s < kSched; ++s) {
+      mbar_init(sfull_bar(s), 1);
+      mbar_init(sempty_bar(s), kRingReaders);
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -764,6 +811,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
   const uint32_t tmem_base = *tmem_slot;
   pdl_prologue();   // the set-up above touched no global memory and may overlap the previous kernel's tail
 
+  // take the next item from this CTA's ring and hand the slot back to the dealer
+  auto ring_take = [&](int &sslot, uint32_t &sphase, int where, int &item) -> bool {
+    if (!mbar_wait_acq_cluster(sfull_bar(sslot), sphase, abort_flag, g.status, where)) return false;
+    item = sched_ring[sslot];
+    return true;
+  };
+  auto ring_release = [&](int &sslot, uint32_t &sphase) {
+    mbar_arrive_remote_plain(mapa_shared(sempty_bar(sslot), 0));
+    if (++sslot == kSched) { sslot = 0; sphase ^= 1u; }
+  };
+
   if (warp == 0 || warp == 6) {
     // ===================== TMA producers (both CTAs): warp 0 loads the A operand, warp 6 the B operand ==========
     // Two threads because one thread issuing every copy of a k-block was close to the critical path.
@@ -774,7 +832,36 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       long long issued = 0;
       bool ok = true;
       const uint32_t full0 = mapa_shared(full_bar(0), 0);
-      for (int item = pair_id; ok && item < g.n_items; item += n_pairs) {
+      const bool dealer = do_a && rank == 0;
+      int sslot = 0;
+      uint32_t sphase = 0;
+      // the dealer: write an item into both CTAs' rings (the slot must have been handed back by all its readers)
+      auto deal = [&](int it) -> bool {
+        if (!mbar_wait(sempty_bar(sslot), sphase ^ 1u, abort_flag, g.status, 410)) return false;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) st_cluster_s32(mapa_shared(ring0 + 4u * sslot, (uint32_t)r), it);
+#pragma unroll
+        for (int r = 0; r < 2; ++r)   // release at cluster scope: the store above is visible to whoever sees this arrival
+          mbar_arrive_cluster(mapa_shared(sfull_bar(sslot), (uint32_t)r));
+        if (++sslot == kSched) { sslot = 0; sphase ^= 1u; }
+        return true;
+      };
+      // it deals one item ahead and draws two ahead, so the counter's round trip is never waited for
+      int item = pair_id, next_item = 0, drawn = 0;
+      if (dealer) {
+        next_item = n_pairs + atomicAdd(&g.status->sched_next, 1);
+        ok = deal(item);
+      }
+      while (ok) {
+        if (dealer) {
+          if (item >= g.n_items) break;   // the end marker has been passed on
+          if (!deal(next_item)) { ok = false; break; }
+          drawn = next_item < g.n_items ? n_pairs + atomicAdd(&g.status->sched_next, 1) : next_item;
+        } else {
+          if (!ring_take(sslot, sphase, 411, item)) { ok = false; break; }
+          ring_release(sslot, sphase);
+          if (item >= g.n_items) break;
+        }
         const Item it = decode_item_pair(g, item);
         const DevProb &q = g.p[it.p];
         const int m0 = it.m0 + (int)rank * 128;          // this CTA's rows of the A operand
@@ -810,6 +897,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
+        if (dealer) { item = next_item; next_item = drawn; }
       }
       if (!ok && rank == 0) {
         long long n = issued < kStages ? issued : kStages;
@@ -827,9 +915,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      int local = 0;
+      int local = 0, sslot = 0;
+      uint32_t sphase = 0;
       bool ok = true;
-      for (int item = pair_id; ok && item < g.n_items; item += n_pairs, ++local) {
+      for (; ok; ++local) {
+        int item;
+        if (!ring_take(sslot, sphase, 510, item)) { ok = false; break; }
+        ring_release(sslot, sphase);
+        if (item >= g.n_items) break;
         const Item it = decode_item_pair(g, item);
         const DevProb &q = g.p[it.p];
         const int nkb = (it.kb1 - it.kb0) + it.next;
@@ -864,9 +957,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
   } else {
     // ===================== epilogue (warps 2..5, both CTAs) =====================
     const int quarter = warp & 3;
-    int local = 0;
+    int local = 0, sslot = 0;
+    uint32_t sphase = 0;
     bool ok = true;
-    for (int item = pair_id; ok && item < g.n_items; item += n_pairs, ++local) {
+    for (; ok; ++local) {
+      int item;
+      ok = __all_sync(0xffffffffu, ring_take(sslot, sphase, 610, item));
+      if (!ok) break;
+      __syncwarp();
+      if (lane == 0) ring_release(sslot, sphase); else if (++sslot == kSched) { sslot = 0; sphase ^= 1u; }
+      __syncwarp();
+      if (item >= g.n_items) break;
       const Item it = decode_item_pair(g, item);
       const DevProb &q = g.p[it.p];
       const int n0 = it.nt * 256;
@@ -896,6 +997,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
                  : "memory");
+  }
+  // the last pair to finish re-arms the item counter for the next launch on this workspace
+  if (rank == 0 && threadIdx.x == 0) {
+    __threadfence();
+    const int done = atomicAdd(&g.status->sched_done, 1);
+    if (done == n_pairs - 1) {
+      g.status->sched_next = 0;
+      g.status->sched_done = 0;
+      __threadfence();
+    }
   }
 }
 
@@ -947,43 +1058,11 @@ __device__ __forceinline__ int4 ld_volatile_i4(const int *p) {
 __device__ __forceinline__ void st_release_gpu(int *p, int v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void st_cluster_s32(uint32_t addr, int v) {
-  asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
 // Remote store of 16 bytes into a peer's shared memory; the peer's mbarrier counts the bytes as they land.
 __device__ __forceinline__ void st_async_v4(uint32_t remote_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
                                             uint32_t remote_bar) {
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
                ::"r"(remote_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar) : "memory");
-}
-// Arrive on a peer's barrier to say "I have finished reading" (nothing of mine needs to become visible).
-__device__ __forceinline__ void mbar_arrive_remote_plain(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_acq_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait whose success also makes a peer's earlier shared-memory stores (released at cluster scope) visible.
-__device__ __noinline__ bool mbar_wait_acq_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                   DeviceStatus *st, int where) {
-  for (int i = 0; i < 4096; ++i)
-    if (mbar_try_acq_cluster(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
-  while (true) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_acq_cluster(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1;
-      if (st && atomicCAS(&st->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) st->where = where;
-      __threadfence();
-      return false;
-    }
-  }
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 

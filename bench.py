@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the dominant kernel (bytes), from an ncu capture summarised under
 # profiles/; valid only while the kernel source is the one that was profiled.
 SHARED_INPUTS = [["q", "k", "v"], ["gate", "up"]]   # projections of a decoder block that read the same tensor
-TRAFFIC = {"tc_gemm_sha1": "b8a8aeb20883793ca0e0004e21d070f2e9fc3b4e", "bytes_per_launch": 1284111488}
+TRAFFIC = {"tc_gemm_sha1": "40d51c0f35237ab99937b748fc9bc0ed34ae6cba", "bytes_per_launch": 1136471808}
 
 
 def load_peaks():

@@ -60,6 +60,26 @@ def test_config1_llama2_7b_block_full(b):
     print("config 1 worst relative errors:", {k: f"{v:.2e}" for k, v in worst.items()})
 
 
+def test_config1_shared_inputs_summed_dx_full(b):
+    # the same block with q,k,v reading one tensor and gate,up another: one summed dX per group
+    from paper_2401_11504_b200 import runtime
+    c = inputs.CONFIGS[1]
+    hp = hp32(inputs.ADAMW)
+    groups = [["q", "k", "v"], ["gate", "up"]]
+    blk = runtime.Block(b, 0, "cfg1s", c["projections"], c["T"], c["r"], c["s"], "bf16", "cuda", input_groups=groups)
+    assert blk.dX[1].data_ptr() == blk.dX[0].data_ptr() and blk.x[2].data_ptr() == blk.x[0].data_ptr()
+    projs0 = snapshot_block(blk)
+    leader = {}
+    for names in groups:
+        for nm in names[1:]:
+            leader[nm] = blk.names.index(names[0])
+    for i, nm in enumerate(blk.names):
+        projs0[i]["dX_to"] = leader.get(nm)
+    _run_update(b, [blk], 1, hp)
+    worst = compare_block(blk, projs0, _oracle_update(projs0, 1, hp), 1, hp["lr"])
+    print("config 1, shared inputs, worst relative errors:", {k: f"{v:.2e}" for k, v in worst.items()})
+
+
 def test_config2_32_blocks_two_epochs(b):
     from paper_2401_11504_b200 import runtime
     c = inputs.CONFIGS[2]

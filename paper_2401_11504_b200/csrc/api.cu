@@ -3,7 +3,6 @@
 #include "common.cuh"
 
 #include <atomic>
-#include <cstdlib>
 #include <cstring>
 #include <utility>
 #include <vector>
@@ -675,83 +674,6 @@ void carve_group(const templora_linear_t *proj, int n, int T, WsAlloc &ws, Group
   }
 }
 
-// The whole pass of a group in ONE launch of the CTA-pair kernel: U and V first (their tiles count up
-// completion counters), y and dX (their rank-r k-blocks wait for U resp. V), dB and dA last (they wait for
-// U resp. V before their first block).  No split-K, no partial slabs, no reductions.
-bool fused_update_ok(int n, void *const *dX) {
-  return use_pairs() && 6 * n <= kTcMaxProblems && getenv("TEMPLORA_FUSE") != nullptr;   // TEMP gate
-}
-templora_status_t update_group_fused(const templora_linear_t *proj, const templora_param_t *As, const templora_param_t *Bs,
-                                     int n, int T, const void *const *x, const void *const *xb, const void *const *dY,
-                                     void *const *y, void *const *dX, const GroupBufs &b, DeviceStatus *status,
-                                     cudaStream_t st) {
-  TcProblem probs[kTcMaxProblems];
-  int np = 0;
-  const int done = 8 * cdiv(T, 256);   // counts of a finished U or V: eight epilogue warps per 256-row tile
-  int owner[kGroup], rank_in_set[kGroup], prob_of[kGroup], max_rank = 0;
-  for (int i = 0; i < n; ++i) {
-    owner[i] = i; rank_in_set[i] = 0; prob_of[i] = -1;
-    if (!(dX && dX[i])) continue;
-    for (int k = 0; k < i && proj[i].input_group != 0; ++k)
-      if (dX[k] && proj[k].input_group == proj[i].input_group) { owner[i] = owner[k]; ++rank_in_set[i]; }
-    if (rank_in_set[i] > max_rank) max_rank = rank_in_set[i];
-  }
-  for (int i = 0; i < n; ++i) {
-    const templora_linear_t *l = proj + i;
-    TcProblem u = prob_U(l, T, xb[i], nullptr, 1);
-    u.out = b.Us[i]; u.out_f32 = 0; u.out_scale = l->s; u.dep_produce = 1 + 2 * i;
-    TcProblem v = prob_V(l, T, dY[i], nullptr, 1);
-    v.out = b.Vs[i]; v.out_f32 = 0; v.out_scale = l->s; v.dep_produce = 2 + 2 * i;
-    probs[np++] = u;
-    probs[np++] = v;
-  }
-  for (int i = 0; i < n; ++i) {
-    const templora_linear_t *l = proj + i;
-    TcProblem py = prob_y(l, T, x[i], b.Us[i], y[i]);
-    py.dep_wait[0] = 1 + 2 * i; py.dep_need[0] = done;
-    probs[np++] = py;
-    if (dX && dX[i]) {
-      if (owner[i] == i) {
-        prob_of[i] = np;
-        TcProblem px = prob_dX(l, T, dY[i], b.Vs[i], dX[i]);
-        if (b.drop[i].xd) px.Kext = 0;   // masked rank-r term: second pass below
-        else { px.dep_wait[0] = 2 + 2 * i; px.dep_need[0] = done; }
-        probs[np++] = px;
-      } else {
-        TcProblem &o = probs[prob_of[owner[i]]];
-        if (l->d_in != proj[owner[i]].d_in || o.n_extra + 2 > 4) return TEMPLORA_ERR_INVALID_ARG;
-        int e = o.n_extra;
-        o.Ax[e] = dY[i]; o.ldax[e] = l->d_out; o.Bx[e] = l->W0; o.ldbx[e] = l->d_in; o.Kx[e] = l->d_out;
-        ++e;
-        if (!b.drop[i].xd) {
-          o.Ax[e] = b.Vs[i]; o.ldax[e] = l->r; o.Bx[e] = l->A; o.ldbx[e] = l->d_in; o.Kx[e] = l->r;
-          ++e;
-          int w = 0;
-          while (w < 3 && o.dep_wait[w] != 0) ++w;
-          if (w == 3) return TEMPLORA_ERR_INVALID_ARG;
-          o.dep_wait[w] = 2 + 2 * i; o.dep_need[w] = done;
-        }
-        o.n_extra = e;
-      }
-    }
-    TcProblem pb = prob_dB(l, T, dY[i], b.Us[i], const_cast<float *>(Bs[i].grad), 1);
-    pb.dep_wait[0] = 1 + 2 * i; pb.dep_need[0] = done; pb.dep_at_start = 1;
-    TcProblem pa = prob_dA(l, T, xb[i], b.Vs[i], const_cast<float *>(As[i].grad), 1);
-    pa.dep_wait[0] = 2 + 2 * i; pa.dep_need[0] = done; pa.dep_at_start = 1;
-    probs[np++] = pb;
-    probs[np++] = pa;
-  }
-  TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, 1));
-  for (int round = 0; round <= max_rank; ++round) {
-    np = 0;
-    for (int i = 0; i < n; ++i)
-      if (dX && dX[i] && b.drop[i].xd && rank_in_set[i] == round)
-        probs[np++] = prob_dX_dropout_term(proj + i, T, b.Vs[i], dX[i], b.drop[i]);
-    if (np) TL_TRY(tc_gemm_grouped(probs, np, 256, status, st, 0));
-  }
-  return TEMPLORA_OK;
-}
-
 templora_status_t update_group_tc(const templora_linear_t *proj, const templora_param_t *As, const templora_param_t *Bs,
                                   int n, int T, const void *const *x, const void *const *dY, void *const *y,
                                   void *const *dX, const GroupBufs &b, DeviceStatus *status, uint64_t steps_taken,
@@ -769,7 +691,6 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
     }
   }
   if (nd) TL_TRY(dropout_apply_batch(drops, nd, st));
-  if (fused_update_ok(n, dX)) return update_group_fused(proj, As, Bs, n, T, x, xb, dY, y, dX, b, status, st);
   for (int i = 0; i < n; ++i) {
     const long long Tr = (long long)T * proj[i].r;
     probs[np++] = prob_U(proj + i, T, xb[i], b.Upart[i], b.su[i]);

@@ -174,14 +174,6 @@ struct TcProblem {
   const void *Ax[4], *Bx[4];
   long long ldax[4], ldbx[4];
   int Kx[4];
-  // plain stores write out_scale * D (0 means 1)
-  float out_scale;
-  // CTA-pair path only: problems of one launch may feed one another.  dep_produce = k > 0: every finished
-  // tile of this problem counts up completion counter k (eight counts per 256 x 256 tile).  dep_wait[e] = k > 0:
-  // this problem's tiles wait until counter k has reached dep_need[e] - before their first k-block
-  // (dep_at_start) or before the first block after the streamed range (their extension and extra pairs read
-  // the producer's output).  Producers are dealt first, so a waiting tile never waits for work not yet started.
-  int dep_produce, dep_wait[3], dep_need[3], dep_at_start;
   // tc_decode_cluster only: role 0 = y of a projection, 1 = its u = A x^T (stored as bf16(epi_scale * u));
   // flag = the projection's index within the launch
   int role, flag;

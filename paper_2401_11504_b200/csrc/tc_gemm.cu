@@ -51,18 +51,10 @@ template <> struct Cfg<64> : CfgBase<64, 8, 128, 1> {};
 template <> struct Cfg<16> : CfgBase<16, 3, 32, 4> {};
 
 constexpr int kMaxExtra = 4;   // further operand pairs accumulated into the same output tile
-constexpr int kMaxDeps = 3;    // problems of the same launch whose outputs a problem may read
-constexpr int kDepCounters = 16;   // completion counters, kept in DeviceStatus::pad[16 ..]
 struct alignas(64) DevProb {
   CUtensorMap tmA, tmB, tmAe, tmBe;
   CUtensorMap tmXa[kMaxExtra], tmXb[kMaxExtra];
   int kb_x[kMaxExtra], kb_xtot;   // k-blocks of each extra pair and their sum (the pairs follow the extension)
-  // pair kernel: problems of one launch that feed one another (see tc_gemm_pair_kernel)
-  int dep_produce;                // completion counter this problem's tiles count up (-1: none)
-  int dep_wait[kMaxDeps], dep_need[kMaxDeps];   // counters to wait for (-1: none) and the counts that mean "complete"
-  int dep_at_start;               // 1: wait before the first k-block, 0: before the first block after the streamed range
-  float out_scale;                // plain stores write out_scale * D
-  int n_mma;                      // pair kernel: width of the MMA, 256, or 64 for problems with N <= 64
   long long out_s0, out_s1, out_split;
   void *out;
   int M, N, kb_main, kb_ext, splits, m_tiles, n_tiles, item_start, a_mn, b_mn, out_f32, pad;
@@ -293,18 +285,17 @@ __device__ __forceinline__ void store_chunk(const DevProb &q, const uint32_t (&v
     }
     return;
   }
-  const float sc = q.out_scale;
   if (q.out_f32) {
     float *o = reinterpret_cast<float *>(q.out) + base;
     if (q.out_s1 == 1 && ncol == NV && ((reinterpret_cast<uintptr_t>(o) & 15) == 0)) {
 #pragma unroll
       for (int c = 0; c < NV; c += 4)
-        *reinterpret_cast<float4 *>(o + c) = make_float4(sc * __uint_as_float(v[c]), sc * __uint_as_float(v[c + 1]),
-                                                         sc * __uint_as_float(v[c + 2]), sc * __uint_as_float(v[c + 3]));
+        *reinterpret_cast<float4 *>(o + c) = make_float4(__uint_as_float(v[c]), __uint_as_float(v[c + 1]),
+                                                         __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
     } else {
 #pragma unroll
       for (int c = 0; c < NV; ++c)
-        if (c < ncol) o[(long long)c * q.out_s1] = sc * __uint_as_float(v[c]);
+        if (c < ncol) o[(long long)c * q.out_s1] = __uint_as_float(v[c]);
     }
   } else {
     __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(q.out) + base;
@@ -312,10 +303,10 @@ __device__ __forceinline__ void store_chunk(const DevProb &q, const uint32_t (&v
 #pragma unroll
       for (int c = 0; c < NV; c += 8) {
         uint4 w;
-        __nv_bfloat162 t0 = __floats2bfloat162_rn(sc * __uint_as_float(v[c]), sc * __uint_as_float(v[c + 1]));
-        __nv_bfloat162 t1 = __floats2bfloat162_rn(sc * __uint_as_float(v[c + 2]), sc * __uint_as_float(v[c + 3]));
-        __nv_bfloat162 t2 = __floats2bfloat162_rn(sc * __uint_as_float(v[c + 4]), sc * __uint_as_float(v[c + 5]));
-        __nv_bfloat162 t3 = __floats2bfloat162_rn(sc * __uint_as_float(v[c + 6]), sc * __uint_as_float(v[c + 7]));
+        __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(v[c]), __uint_as_float(v[c + 1]));
+        __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+        __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[c + 4]), __uint_as_float(v[c + 5]));
+        __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(v[c + 6]), __uint_as_float(v[c + 7]));
         w.x = *reinterpret_cast<uint32_t *>(&t0);
         w.y = *reinterpret_cast<uint32_t *>(&t1);
         w.z = *reinterpret_cast<uint32_t *>(&t2);
@@ -325,7 +316,7 @@ __device__ __forceinline__ void store_chunk(const DevProb &q, const uint32_t (&v
     } else {
 #pragma unroll
       for (int c = 0; c < NV; ++c)
-        if (c < ncol) o[(long long)c * q.out_s1] = __float2bfloat16_rn(sc * __uint_as_float(v[c]));
+        if (c < ncol) o[(long long)c * q.out_s1] = __float2bfloat16_rn(__uint_as_float(v[c]));
     }
   }
 }
@@ -652,11 +643,6 @@ __global__ void __launch_bounds__(kThreads2, 1) tc_gemm_kernel(const __grid_cons
 }
 
 // ------------------------------------------------------------------ helpers shared by the cluster kernels
-__device__ __forceinline__ int ld_volatile_s32(const int *p) {
-  int v;
-  asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
 __device__ __forceinline__ void st_cluster_s32(uint32_t addr, int v) {
   asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -745,9 +731,9 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ uint32_t instr_desc_pair(int a_mn, int b_mn, int n) {  // M = 256, N = n
+__device__ __forceinline__ uint32_t instr_desc_pair(int a_mn, int b_mn) {  // M = 256, N = 256
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+         ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
 // item -> (problem, 256-row tile, 256-column tile); no split-K on this path
@@ -791,7 +777,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
   constexpr int kRingReaders = 12;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int *dep_cnt = &g.status->pad[16];            // completion counters of problems that feed others (zero between launches)
   const uint32_t rank = cluster_ctarank();      // 0: issues the MMAs; 1: its peer
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
@@ -848,7 +833,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       bool ok = true;
       const uint32_t full0 = mapa_shared(full_bar(0), 0);
       const bool dealer = do_a && rank == 0;
-      uint32_t deps_ready = 0;   // completion counters this thread has seen complete
       int sslot = 0;
       uint32_t sphase = 0;
       // the dealer: write an item into both CTAs' rings (the slot must have been handed back by all its readers)
@@ -880,45 +864,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
         }
         const Item it = decode_item_pair(g, item);
         const DevProb &q = g.p[it.p];
-        bool deps_pending = q.dep_wait[0] >= 0;
-        // The operands named by the extension and extra pairs (or, with dep_at_start, all operands) are written by
-        // other tiles of this launch: wait (bounded) until their completion counters say they are whole.
-        auto wait_deps = [&]() -> bool {
-          const unsigned long long t0 = globaltimer_ns();
-          for (int e = 0; e < kMaxDeps; ++e) {
-            const int c = q.dep_wait[e];
-            if (c < 0 || ((deps_ready >> c) & 1u)) continue;
-            while (ld_volatile_s32(dep_cnt + c) < q.dep_need[e]) {
-              if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                if (atomicCAS(&g.status->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) g.status->where = 420;
-                __threadfence();
-                return false;
-              }
-            }
-            deps_ready |= 1u << c;
-          }
-          __threadfence();                                      // acquire side of the counters
-          asm volatile("fence.proxy.async;" ::: "memory");      // those generic-proxy writes are read by TMA below
-          return true;
-        };
-        if (deps_pending && q.dep_at_start) {
-          if (!wait_deps()) { ok = false; break; }
-          deps_pending = false;
-        }
         const int m0 = it.m0 + (int)rank * 128;          // this CTA's rows of the A operand
-        // this CTA's half of the B operand: 128 columns of a 256-wide tile, or 32 of a 64-wide one (the copy still
-        // fetches a 128-row box; the MMA reads its first 32 rows or columns)
-        const int n0 = q.n_mma == 64 ? (int)rank * 32 : it.nt * 256 + (int)rank * 128;
+        const int n0 = it.nt * 256 + (int)rank * 128;    // this CTA's half of the B operand
         const int pa_mn = q.a_mn, pb_mn = q.b_mn;
         const int nmain = it.kb1 - it.kb0;
         const int nkb = nmain + it.next;
         KCursor cur(q, it.kb0, nmain);
         for (int i = 0; i < nkb; ++i) {
-          if (deps_pending && i == nmain) {
-            if (!wait_deps()) { ok = false; break; }
-            deps_pending = false;
-          }
           const CUtensorMap *ma, *mb;
           int kel;
           cur.take(ma, mb, kel);
@@ -980,7 +932,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 256);
         const int a_mn = q.a_mn, b_mn = q.b_mn;
-        const uint32_t idesc = instr_desc_pair(a_mn, b_mn, q.n_mma);
+        const uint32_t idesc = instr_desc_pair(a_mn, b_mn);
         const uint64_t a_tmpl = smem_desc_template(a_mn), b_tmpl = smem_desc_template(b_mn);
         const uint32_t a_step = smem_desc_kstep(a_mn), b_step = smem_desc_kstep(b_mn);
         for (int i = 0; i < nkb; ++i) {
@@ -1027,7 +979,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 256);
       uint32_t v[32];
 #pragma unroll 1
-      for (int c0 = 0; c0 < q.n_mma; c0 += 32) {
+      for (int c0 = 0; c0 < 256; c0 += 32) {
         tmem_ld32(t_row + c0, v);
         tmem_ld_wait();
         store_chunk<32>(q, v, row, n0 + c0, 0);
@@ -1035,12 +987,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
-      if (q.dep_produce >= 0) {   // this warp's rows of the tile are written: count them in
-        __threadfence();
-        asm volatile("fence.proxy.async;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) atomicAdd(dep_cnt + q.dep_produce, 1);
-      }
     }
   }
 
@@ -1059,7 +1005,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     if (done == n_pairs - 1) {
       g.status->sched_next = 0;
       g.status->sched_done = 0;
-      for (int c = 0; c < kDepCounters; ++c) dep_cnt[c] = 0;
       __threadfence();
     }
   }
@@ -1726,8 +1671,7 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
   if (!di || di->cc_major != 10) return TEMPLORA_ERR_UNSUPPORTED;
   if (!status) return TEMPLORA_ERR_WORKSPACE;  // the kernel keeps its item counter in the status record
 
-  // problems whose outputs others of this launch read come first (a waiting tile then never waits for work
-  // that has not started), then heaviest work items first, so that the schedule ends on the short ones
+  // heaviest work items first: the static round-robin schedule then ends on the short ones
   int order[kTcMaxProblems];
   for (int i = 0; i < n; ++i) order[i] = i;
   auto weight = [&](int i) {
@@ -1736,7 +1680,6 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     int s = p.splits < 1 ? 1 : p.splits;
     long long w = (kb + s - 1) / s + (p.Kext + BK - 1) / BK;
     for (int e = 0; e < p.n_extra; ++e) w += (p.Kx[e] + BK - 1) / BK;
-    if (p.dep_produce > 0) w += 1LL << 40;
     return w;
   };
   for (int i = 1; i < n; ++i)
@@ -1780,17 +1723,6 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
       q.tmAe = q.tmA;
       q.tmBe = q.tmB;
     }
-    q.out_scale = p.out_scale == 0.f ? 1.f : p.out_scale;
-    q.n_mma = (use_pair && p.N <= 64 && !p.epi_mask) ? 64 : 256;
-    q.dep_produce = p.dep_produce - 1;
-    q.dep_at_start = p.dep_at_start;
-    for (int e = 0; e < kMaxDeps; ++e) {
-      q.dep_wait[e] = p.dep_wait[e] - 1;
-      q.dep_need[e] = p.dep_need[e];
-      if (p.dep_wait[e] < 0 || p.dep_wait[e] > kDepCounters) return TEMPLORA_ERR_INVALID_ARG;
-      if (p.dep_wait[e] && !use_pair) return TEMPLORA_ERR_UNSUPPORTED;
-    }
-    if (p.dep_produce < 0 || p.dep_produce > kDepCounters || (p.dep_produce && !use_pair)) return TEMPLORA_ERR_INVALID_ARG;
     q.kb_xtot = 0;
     if (p.n_extra < 0 || p.n_extra > kMaxExtra || (p.n_extra > 0 && q.splits > 1)) return TEMPLORA_ERR_INVALID_ARG;
     for (int e = 0; e < kMaxExtra; ++e) {
@@ -1846,9 +1778,7 @@ templora_status_t tc_decode_cluster(const TcProblem *probs, int n, int n_tokens,
     q.a_mn = 0; q.b_mn = 0; q.out_f32 = 0;
     q.pad = p.role; q.pad3 = p.flag;
     q.kb_xtot = 0;
-    for (int e = 0; e < kMaxExtra; ++e) q.kb_x[e] = 0;
-    q.out_scale = 1.f; q.n_mma = 256; q.dep_produce = -1; q.dep_at_start = 0;
-    for (int e = 0; e < kMaxDeps; ++e) { q.dep_wait[e] = -1; q.dep_need[e] = 0; }
+    for (int e = 0; e < kMaxExtra; ++e) { q.kb_x[e] = 0; q.tmXa[e] = q.tmA; q.tmXb[e] = q.tmB; }
     q.epi_mask = nullptr; q.epi_mask_pitch = 0; q.epi_scale = p.epi_scale;
     q.out = p.out; q.out_s0 = 1; q.out_s1 = p.out_s1; q.out_split = 0;
     items += q.m_tiles;

@@ -478,3 +478,27 @@ def test_shared_dx_needs_equal_input_width(b):
     args = b.UpdateBlockArgs(lins, As, Bs, [d["x"] for d in devs], [d["dY"] for d in devs], ys, [dX, dX])
     with pytest.raises(b.TemploraError):
         b.templora_update_block(args, 1, 1e-4, 0.9, 0.999, 1e-8, 0.0, 0, ws)
+
+
+def test_decode_block_under_a_tight_sm_cap(b):
+    # eight SMs fit fewer clusters than the call has projections: the one-kernel form steps aside for the
+    # two-kernel form, and a cap of 24 SMs runs the one-kernel form on few clusters; both must match
+    shapes = [(512, 640, 64)] * 4 + [(1024, 384, 64)] * 3
+    n = 4
+    hosts = [inputs.make_linear(37, f"cap-{i}", n, di, do, r, dtype="bf16") for i, (di, do, r) in enumerate(shapes)]
+    devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
+    lins = [b.linear_desc(d["W0"], d["A"], d["B"], 2.0) for d in devs]
+    ws = b.alloc_workspace(b.templora_decode_block_workspace_bytes(lins))
+    stream = torch.cuda.Stream()
+    for cap in (8, 24, 0):
+        b.templora_set_stream_sm_limit(stream, cap)
+        ys = [torch.full((n, do), float("nan"), dtype=torch.bfloat16, device="cuda") for _, do, _ in shapes]
+        args = b.DecodeBlockArgs(lins, [d["x"] for d in devs], ys)
+        torch.cuda.synchronize()
+        b.templora_decode_block_fwd(args, ws, stream=stream)
+        stream.synchronize()
+        assert b.templora_read_device_status(ws, stream=stream)[0] == 0
+        for i, h in enumerate(hosts):
+            ref = orc.decode_fwd(f64(h["x"]), f64(h["W0"]), f64(h["A"]), f64(h["B"]), 2.0)
+            assert_close(f"cap {cap} y{i}", f64(ys[i]), ref, TOL["bf16"])
+    b.templora_set_stream_sm_limit(stream, 0)

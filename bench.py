@@ -243,7 +243,7 @@ def run_ours(args):
     achieved = flops_main / (ms_main / n_main * 1e-3) / 1e12 if n_main else None
     sha = kernel_sha1()
     traffic = TRAFFIC["bytes_per_launch"] if (TRAFFIC["tc_gemm_sha1"] == sha and default_workload) else None
-    roofline = {"bound": "tensor", "kernel": "tc_gemm_kernel<256> (y and dX of 7 projections, rank-r terms fused)",
+    roofline = {"bound": "tensor", "kernel": "pair::tc_gemm_pair_kernel (y and dX of every projection of the block, rank-r terms fused)",
                 "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
                 "frac": (achieved / peaks["tflops"]) if achieved else None, "traffic": traffic,
                 "peak_source": f"{peaks['source']}: cuBLAS bf16 sustained (kernel timed inside a long step); burst {peaks['burst']}",

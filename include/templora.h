@@ -298,12 +298,17 @@ int32_t templora_set_kernel_path(int32_t mode);
  *     (the call clears the part that must start at zero).  Two calls that may overlap on the
  *     GPU, e.g. on different streams, race on it: serialise them, or use templora_decode_fwd
  *     with one workspace per stream.
- *   - The device status record of this variant lives in the array and is cleared at the start
- *     of each call; templora_read_device_status cannot reach it.
+ *   - Arguments are checked as in templora_decode_fwd before anything is enqueued; a refused
+ *     call leaves the array untouched.
+ *   - The device status record of this variant lives at the head of the array and is cleared
+ *     when an accepted call starts, so it describes the most recent call only.  Read it with
+ *     templora_decode_fwd_noalloc_status, which does what templora_read_device_status does
+ *     (synchronises `stream`, copies the record out) and allocates nothing either.
  */
 #define TEMPLORA_NOALLOC_SCRATCH_BYTES (8u << 20)
 templora_status_t templora_decode_fwd_noalloc(const templora_linear_t *lin, int32_t n_tokens, const void *x,
                                               void *y, void *stream);
+templora_status_t templora_decode_fwd_noalloc_status(void *stream, int32_t *code, int32_t *where);
 
 /*
  * Launch accounting, a profiling aid (the paper has no counterpart).  The library counts

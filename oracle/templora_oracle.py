@@ -34,7 +34,11 @@ integer worked example under tests/golden/, B = 0 reduction, the merged-weight
 identity, exact finite differences (the loss sum(dY*y) is linear in each of
 x, A, B separately), additivity of dA/dB over row partitions, the closed-form
 first AdamW step, the constant-gradient AdamW trajectory, and torch's own
-bfloat16 cast for the rounding helper.
+bfloat16 cast for the rounding helper.  The dropout mask: the generator against
+its published known-answer vectors, and the element -> (counter, word) layout
+against a hand case built from the first of those vectors and against a scalar
+restatement of the rule with 64-bit seeds and offsets and rows that start inside
+a block.
 
 Parity with numbers printed by the paper: parity unpinned.  The paper prints no
 worked numeric example and no per-layer value for this path; the pins above are
@@ -178,7 +182,7 @@ def lr_at_step(lr, step, warmup_steps):
 
 
 def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf16_work=False, batch=None,
-                 dropout_p=0.0, warmup_steps=0, lr_round=None):
+                 dropout_p=0.0, warmup_steps=0, lr_round=None, grad_log=None):
     """projs: list of dicts with keys x, dY, W0, s, A_master, B_master and optionally
     mA, vA, mB, vB (default 0).  For each epoch: forward and backward of every
     projection with the current working A, B; then step += 1 and AdamW on every
@@ -199,6 +203,9 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
     With warmup_steps > 0 the step numbered k (step0 + 1, step0 + 2, ...) uses lr_at_step(lr, k,
     warmup_steps); lr_round, if given, is applied to that rate (the tests pass the fp32 rounding
     that the C ABI's float argument imposes).
+
+    grad_log, if a list, receives one entry (step, projection index, dA, dB) per projection and optimizer
+    step: the gradients that step's AdamW consumed (a record for the tests; it changes nothing computed).
 
     Returns (state, step): state[i] has A_master, B_master, mA, vA, mB, vB and the
     last epoch's y, dX, dA, dB.
@@ -234,6 +241,8 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
                 else:
                     st[p["dX_to"]]["dX"][rows] += dXb
             step += 1
+            if grad_log is not None:
+                grad_log.extend((step, i, q["dA"].copy(), q["dB"].copy()) for i, q in enumerate(st))
             lr_k = lr_at_step(lr, step, warmup_steps)
             if lr_round is not None:
                 lr_k = lr_round(lr_k)

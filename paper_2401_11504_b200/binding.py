@@ -24,7 +24,7 @@ EXPORTS = [
     "templora_decode_block_workspace_bytes", "templora_decode_block_fwd", "templora_update_block_batched",
     "templora_set_stream_sm_limit", "templora_selftest_bounded_wait", "templora_lr_at_step",
     "templora_update_block_warmup", "templora_swiglu_fwd", "templora_swiglu_bwd", "templora_rmsnorm_fwd",
-    "templora_rmsnorm_bwd",
+    "templora_rmsnorm_bwd", "templora_decode_fwd_noalloc_status",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 (KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
@@ -104,6 +104,8 @@ def _load():
     lib.templora_decode_block_fwd.argtypes = [LP, i32, i32, C.POINTER(vp), C.POINTER(vp), vp, sz, vp]
     lib.templora_decode_fwd_noalloc.restype = i32
     lib.templora_decode_fwd_noalloc.argtypes = [LP, i32, vp, vp, vp]
+    lib.templora_decode_fwd_noalloc_status.restype = i32
+    lib.templora_decode_fwd_noalloc_status.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
     lib.templora_timing_enable.restype = None
     lib.templora_timing_enable.argtypes = [i32]
     lib.templora_timing_read.restype = i32
@@ -314,6 +316,14 @@ def templora_decode_fwd_noalloc(lin, x, y, stream=None):
     all calls on the device, so calls that could overlap on the GPU must be serialised."""
     _check(lib.templora_decode_fwd_noalloc(C.byref(lin), x.shape[0], _ptr(x), _ptr(y), _stream(stream)),
            "templora_decode_fwd_noalloc")
+
+
+def templora_decode_fwd_noalloc_status(stream=None):
+    """(code, where) of the most recent templora_decode_fwd_noalloc call on this device; synchronises the stream."""
+    code, where = C.c_int32(0), C.c_int32(0)
+    _check(lib.templora_decode_fwd_noalloc_status(_stream(stream), C.byref(code), C.byref(where)),
+           "templora_decode_fwd_noalloc_status")
+    return code.value, where.value
 
 
 def templora_decode_block_workspace_bytes(lins):

@@ -875,6 +875,14 @@ size_t decode_workspace_need(const templora_linear_t *lin, int n) {
   return need;
 }
 
+templora_status_t decode_check_args(const templora_linear_t *lin, int n_tokens, const void *x, const void *y) {
+  TL_TRY(check_linear(lin));
+  TL_TRY(check_linear_ptrs(lin));
+  if (n_tokens < 1 || n_tokens > 16) return TEMPLORA_ERR_INVALID_ARG;
+  if (!x || !y || !aligned16(x) || !aligned16(y)) return TEMPLORA_ERR_INVALID_ARG;
+  return TEMPLORA_OK;
+}
+
 }  // namespace templora
 
 using namespace templora;
@@ -960,10 +968,7 @@ templora_status_t templora_adamw_step(const templora_param_t *params, int32_t n_
 
 templora_status_t templora_decode_fwd(const templora_linear_t *lin, int32_t n_tokens, const void *x, void *y, void *ws,
                                       size_t ws_bytes, void *stream) {
-  TL_TRY(check_linear(lin));
-  TL_TRY(check_linear_ptrs(lin));
-  if (n_tokens < 1 || n_tokens > 16) return TEMPLORA_ERR_INVALID_ARG;
-  if (!x || !y || !aligned16(x) || !aligned16(y)) return TEMPLORA_ERR_INVALID_ARG;
+  TL_TRY(decode_check_args(lin, n_tokens, x, y));
   TL_TRY(check_ws(ws, ws_bytes));
   WsAlloc a(ws, ws_bytes);
   return decode_impl(lin, n_tokens, x, y, a, false, reinterpret_cast<cudaStream_t>(stream));

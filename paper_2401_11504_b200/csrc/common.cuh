@@ -195,5 +195,7 @@ templora_status_t tc_wait_selftest(DeviceStatus *status, unsigned long long limi
 
 // ---- workspace need of the decode-time forward alone (api.cu) -------------------
 size_t decode_workspace_need(const templora_linear_t *lin, int n);
+// The argument checks of templora_decode_fwd that do not involve the workspace.
+templora_status_t decode_check_args(const templora_linear_t *lin, int n_tokens, const void *x, const void *y);
 
 }  // namespace templora

@@ -46,9 +46,10 @@ using namespace templora;
 
 extern "C" templora_status_t templora_decode_fwd_noalloc(const templora_linear_t *lin, int32_t n_tokens, const void *x,
                                                          void *y, void *stream) {
-  if (!lin) return TEMPLORA_ERR_INVALID_ARG;
+  // every argument check of templora_decode_fwd runs first: a refused call enqueues nothing and leaves the
+  // status record of the previous call in place
+  TL_TRY(decode_check_args(lin, n_tokens, x, y));
   // reject shapes whose partial sums do not fit the built-in array before touching the device
-  if (n_tokens < 1 || n_tokens > 16) return TEMPLORA_ERR_INVALID_ARG;
   const size_t need = decode_workspace_need(lin, n_tokens);
   if (need == 0) return TEMPLORA_ERR_INVALID_ARG;
   if (need > kNoAllocBytes) return TEMPLORA_ERR_UNSUPPORTED;
@@ -58,4 +59,12 @@ extern "C" templora_status_t templora_decode_fwd_noalloc(const templora_linear_t
   // start at zero; the partial sums are fully rewritten before they are read.
   TL_CUDA_CHECK(cudaMemsetAsync(scratch, 0, kStatusBytes, reinterpret_cast<cudaStream_t>(stream)));
   return templora_decode_fwd(lin, n_tokens, x, y, scratch, kNoAllocBytes, stream);
+}
+
+extern "C" templora_status_t templora_decode_fwd_noalloc_status(void *stream, int32_t *code, int32_t *where) {
+  if (!code || !where) return TEMPLORA_ERR_INVALID_ARG;
+  void *scratch = nullptr;
+  TL_TRY(scratch_for_current_device(&scratch));
+  // same steps as templora_read_device_status, aimed at the head of the built-in array
+  return templora_read_device_status(scratch, stream, code, where);
 }

@@ -110,9 +110,47 @@ def snapshot_block(blk):
     return projs
 
 
-def compare_block(blk, projs0, ref, epochs, lr, tol=1e-2, check_io=True):
-    """Device state of a block after templora_update_block against the oracle's update_block."""
+def small_gradient_mask(grad_log, i, nm, tol):
+    """Elements of projection i's A (or B) whose reference gradient lies, in at least one optimizer step, within the
+    gradient's own tolerance of zero: |g| <= tol * max|g| of that step.  grad_log is what oracle.update_block
+    recorded.  Adam's step is sign-like there (lr * g / (|g| + eps) at the first step), so the two sides may
+    legitimately take different steps on these elements, and on these only."""
+    mask = None
+    for _, j, dA, dB in grad_log:
+        if j != i:
+            continue
+        g = np.abs(dA if nm == "A" else dB)
+        small = g <= tol * g.max()
+        mask = small if mask is None else (mask | small)
+    assert mask is not None, "no gradients recorded for this projection"
+    return mask
+
+
+def check_adam_steps(name, p0, got, ref, small_g, tol, n_steps, lr, max_frac=0.02):
+    """The optimizer's movement got - p0 against the oracle's ref - p0 (|movement| ~ n_steps * lr << |p|, so a check
+    on p alone would pass a kernel that does nothing).  Tight bound: tol * max|movement| plus one fp32 ulp of p.
+    Elements outside it must all be ones whose gradient is within tolerance of zero (small_g), must stay within
+    the worst case of a sign flip (2 lr per step), and must be few.  Returns their fraction."""
+    assert np.isfinite(got).all(), f"{name}: non-finite master parameters"
+    d_gpu, d_ref = got - p0, ref - p0
+    assert np.abs(d_ref).max() > 0, f"{name}: the oracle did not move the parameters"
+    bound = tol * np.abs(d_ref).max() + 2.0 ** -23 * np.abs(ref).max()
+    dev = np.abs(d_gpu - d_ref)
+    off = dev > bound
+    unexplained = off & ~small_g
+    assert not unexplained.any(), (f"{name}: {int(unexplained.sum())} optimizer steps are off by up to "
+                                   f"{dev[unexplained].max():.3e} (bound {bound:.3e}) where the gradient is not small")
+    assert dev.max() <= 2.0 * n_steps * lr * (1.0 + 1e-3) + bound, f"{name}: a step is off by more than a sign flip"
+    frac = float(off.mean())
+    assert frac <= max_frac, f"{name}: {frac:.4f} of the optimizer steps are off"
+    return frac
+
+
+def compare_block(blk, projs0, ref, epochs, lr, tol=1e-2, check_io=True, grad_log=None):
+    """Device state of a block after templora_update_block against the oracle's update_block.  `epochs` is the
+    number of optimizer steps taken; grad_log the per-step gradients recorded by the oracle."""
     worst = {}
+    fracs = {}
     for i, (q, st) in enumerate(zip(ref, blk.state)):
         name = blk.names[i]
         if check_io:
@@ -124,14 +162,11 @@ def compare_block(blk, projs0, ref, epochs, lr, tol=1e-2, check_io=True):
         for nm in ("A", "B"):
             p0 = projs0[i][nm + "_master"]
             got = f64(st[nm]["master"])
-            err = np.abs(got - q[nm + "_master"]).max()
-            assert err <= tol * np.abs(q[nm + "_master"]).max() + 2.0 * epochs * lr, f"{name}.{nm} master"
-            d_gpu, d_ref = got - p0, q[nm + "_master"] - p0
-            assert np.abs(d_ref).max() > 0
-            bound = tol * np.abs(d_ref).max() + 2.0 ** -23 * np.abs(q[nm + "_master"]).max()
-            frac = (np.abs(d_gpu - d_ref) > bound).mean()
-            assert frac <= 0.02, f"{name}.{nm}: {frac:.4f} of the optimizer steps are off"
+            fracs[f"{name}.{nm}"] = check_adam_steps(f"{name}.{nm}", p0, got, q[nm + "_master"],
+                                                     small_gradient_mask(grad_log, i, nm, tol), tol, epochs, lr)
             assert_close(f"{name}.m{nm}", f64(st[nm]["m"]), q["m" + nm], tol)
             assert_close(f"{name}.v{nm}", f64(st[nm]["v"]), q["v" + nm], 2 * tol)
             assert np.array_equal(f64(st[nm]["work"]), orc.round_bf16(got.astype(np.float32))), f"{name}.{nm} work copy"
+    print("fraction of optimizer steps outside the tight bound (all at gradients within tolerance of zero):",
+          {k: f"{v:.4f}" for k, v in fracs.items()})
     return worst

@@ -60,6 +60,29 @@ def test_workspace_sizes_are_sane(b):
     assert b.templora_update_block_workspace_bytes(lins * 32, 1024) <= 2 * nb
 
 
+def test_noalloc_scratch_holds_every_7b_and_70b_projection(b):
+    # the header promises that the built-in array of templora_decode_fwd_noalloc is large enough for every
+    # Llama-2 7B- and 70B-shaped projection at rank 64 with up to 16 tokens, in either decode kernel form
+    from paper_2401_11504_b200 import inputs
+    lib = b.lib
+    assert b.NOALLOC_SCRATCH_BYTES == 8 << 20
+    worst = 0
+    for block in (inputs.LLAMA2_7B_BLOCK, inputs.LLAMA2_70B_BLOCK):
+        for name, d_in, d_out in block:
+            need = b.templora_decode_block_workspace_bytes([_lin(b, d_in, d_out, 64)])
+            assert 1024 <= need <= b.NOALLOC_SCRATCH_BYTES, (name, d_in, d_out, need)
+            worst = max(worst, need)
+    assert worst > (1 << 20)     # the query really measures the split-K slabs, not just the head
+    # refusals need no GPU: token count, rank, missing tensors
+    lin = _lin(b)
+    vp = C.c_void_p
+    assert lib.templora_decode_fwd_noalloc(C.byref(lin), 17, vp(0x1000), vp(0x1000), None) == b.ERR_INVALID_ARG
+    assert lib.templora_decode_fwd_noalloc(C.byref(lin), 4, None, vp(0x1000), None) == b.ERR_INVALID_ARG
+    assert lib.templora_decode_fwd_noalloc(C.byref(_lin(b, r=257)), 4, vp(0x1000), vp(0x1000), None) == b.ERR_UNSUPPORTED
+    assert lib.templora_decode_fwd_noalloc(C.byref(_lin(b, 64, 1 << 18, 8)), 16, vp(0x1000), vp(0x1000), None) == b.ERR_UNSUPPORTED
+    assert lib.templora_decode_fwd_noalloc_status(None, None, None) == b.ERR_INVALID_ARG
+
+
 def test_argument_errors_are_synchronous(b):
     lib = b.lib
     lin = _lin(b)

@@ -394,6 +394,113 @@ def test_dropout_keep_statistics_and_determinism():
     assert orc.dropout_keep(9, 0, 4, 16, 0.3).shape == (4, 16)
 
 
+# A scalar restatement of the generator and of the mask rule, in plain Python integers, sharing nothing
+# with the oracle's vectorised code.  The generator is checked against its published vectors below
+# before it is used as a yardstick.
+_KAT = [
+    ((0, 0, 0, 0), (0, 0), (0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8)),
+    ((0xffffffff,) * 4, (0xffffffff, 0xffffffff), (0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd)),
+    ((0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344), (0xa4093822, 0x299f31d0),
+     (0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1)),
+]
+
+
+def _philox_scalar(ctr, key):
+    c0, c1, c2, c3 = ctr
+    k0, k1 = key
+    for _ in range(10):
+        lo0, hi0 = (0xD2511F53 * c0) & 0xFFFFFFFF, (0xD2511F53 * c0) >> 32
+        lo1, hi1 = (0xCD9E8D57 * c2) & 0xFFFFFFFF, (0xCD9E8D57 * c2) >> 32
+        c0, c1, c2, c3 = hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0
+        k0, k1 = (k0 + 0x9E3779B9) & 0xFFFFFFFF, (k1 + 0xBB67AE85) & 0xFFFFFFFF
+    return (c0, c1, c2, c3)
+
+
+def _keep_by_rule(seed, offset, T, d_in, p):
+    """The mask rule of the library's header, element by element: element e = t*d_in + k takes word e % 4 of
+    the block whose counter is (lo(e/4), hi(e/4), lo(offset), hi(offset)) under key (lo(seed), hi(seed));
+    dropped iff that word < floor(p * 2^32)."""
+    thr = int(math.floor(p * 4294967296.0))
+    lo, hi = (lambda v: v & 0xFFFFFFFF), (lambda v: (v >> 32) & 0xFFFFFFFF)
+    keep = np.zeros((T, d_in), dtype=np.uint8)
+    for t in range(T):
+        for k in range(d_in):
+            e = t * d_in + k
+            word = _philox_scalar((lo(e // 4), hi(e // 4), lo(offset), hi(offset)), (lo(seed), hi(seed)))[e % 4]
+            keep[t, k] = 0 if word < thr else 1
+    return keep
+
+
+def _dropout_layout_pins_pass(keep_fn):
+    try:
+        # (1) first published vector: counter (0,0,0,0), key (0,0) -> 6627e8d5 e169c58d bc57ac4c 9b00dbd8.
+        #     seed 0, offset 0, one row of four elements, p = 0.5 (threshold 0x80000000): only the first
+        #     word is below the threshold, so element 0 is dropped and elements 1..3 are kept.
+        ok = np.array_equal(keep_fn(0, 0, 1, 4, 0.5), np.array([[0, 1, 1, 1]], dtype=np.uint8))
+        #     same draws against p = 0.75 (0xC0000000): 66.. 9b.. bc.. are below, e1.. is not.
+        ok = ok and np.array_equal(keep_fn(0, 0, 1, 4, 0.75), np.array([[0, 1, 0, 0]], dtype=np.uint8))
+        # (2) a 64-bit offset and a 64-bit seed whose low and high words differ, rows of 6 elements so that
+        #     rows 1 and 2 start in the middle of a block (e = 6 -> block 1 word 2; e = 12 -> block 3 word 0),
+        #     and 18 elements = four full blocks and a half
+        seed, offset = 0x0123456789ABCDEF, 0x00000002_00000005
+        for p in (0.5, 0.3):
+            ok = ok and np.array_equal(keep_fn(seed, offset, 3, 6, p), _keep_by_rule(seed, offset, 3, 6, p))
+        # (3) the step offset enters the counter, not the key: offset 1 with seed 0 is a different block
+        #     from offset 0 with seed 1
+        ok = ok and np.array_equal(keep_fn(0, 1, 2, 8, 0.5), _keep_by_rule(0, 1, 2, 8, 0.5))
+        ok = ok and np.array_equal(keep_fn(1, 0, 2, 8, 0.5), _keep_by_rule(1, 0, 2, 8, 0.5))
+        return bool(ok)
+    except Exception:
+        return False
+
+
+def test_dropout_keep_layout_by_hand_and_by_scalar_rule():
+    for ctr, key, want in _KAT:                    # the yardstick itself against the published vectors
+        assert _philox_scalar(ctr, key) == want
+    # the scalar rule reproduces the hand case too (so the yardstick's word order is the header's)
+    assert np.array_equal(_keep_by_rule(0, 0, 1, 4, 0.5), [[0, 1, 1, 1]])
+    assert _dropout_layout_pins_pass(orc.dropout_keep)
+    # the cases of (2) are not degenerate: both values occur, and the 64-bit halves matter
+    m = _keep_by_rule(0x0123456789ABCDEF, 0x00000002_00000005, 3, 6, 0.5)
+    assert 0 < m.sum() < m.size
+    assert not np.array_equal(m, _keep_by_rule(0x0123456789ABCDEF, 0x00000005_00000002, 3, 6, 0.5))
+    assert not np.array_equal(m, _keep_by_rule(0x89ABCDEF01234567, 0x00000002_00000005, 3, 6, 0.5))
+
+
+def test_dropout_layout_pins_catch_planted_mistakes():
+    """Copies of the oracle's mask routine with one layout mistake each must fail the pins above."""
+    def variant(kind):
+        def fn(seed, offset, T, d_in, p):
+            seed, offset = int(seed), int(offset)
+            n = T * d_in
+            lo, hi = (lambda v: v & 0xFFFFFFFF), (lambda v: (v >> 32) & 0xFFFFFFFF)
+            key = (lo(seed), hi(seed))
+            if kind == "key_halves_swapped": key = (hi(seed), lo(seed))
+            thr = min(orc.dropout_threshold(p), 0xFFFFFFFF)
+            out = np.zeros(n, dtype=np.uint8)
+            for e in range(n):
+                blk, word = e // 4, e % 4
+                if kind == "rows_start_new_blocks":
+                    t, k = divmod(e, d_in)
+                    blk, word = t * ((d_in + 3) // 4) + k // 4, k % 4
+                ctr = [lo(blk), hi(blk), lo(offset), hi(offset)]
+                if kind == "offset_halves_swapped": ctr = [lo(blk), hi(blk), hi(offset), lo(offset)]
+                if kind == "offset_in_words_0_1": ctr = [lo(offset), hi(offset), lo(blk), hi(blk)]
+                if kind == "offset_added_to_index": ctr = [lo(blk + offset), hi(blk + offset), 0, 0]
+                if kind == "offset_in_key": ctr, key = [lo(blk), hi(blk), 0, 0], (lo(seed + offset), hi(seed + offset))
+                if kind == "words_reversed": word = 3 - word
+                if kind == "one_block_per_element": ctr, word = [lo(e), hi(e), lo(offset), hi(offset)], 0
+                draw = int(orc.philox4x32_10(np.array([ctr], dtype=np.uint32), key)[0][word])
+                out[e] = (draw >= thr) if kind != "keeps_below_threshold" else (draw < thr)
+            return out.reshape(T, d_in)
+        return fn
+    assert _dropout_layout_pins_pass(variant("none"))    # the copy without a mistake passes
+    for kind in ("key_halves_swapped", "rows_start_new_blocks", "offset_halves_swapped", "offset_in_words_0_1",
+                 "offset_added_to_index", "offset_in_key", "words_reversed", "one_block_per_element",
+                 "keeps_below_threshold"):
+        assert not _dropout_layout_pins_pass(variant(kind)), kind
+
+
 def test_dropout_forward_backward_against_loops_and_differences():
     T, d_in, d_out, r, s, p = 5, 8, 6, 3, 2.0, 0.25
     x, W0, A, B, dY = rnd(T, d_in), rnd(d_out, d_in), rnd(r, d_in), rnd(d_out, r), rnd(T, d_out)

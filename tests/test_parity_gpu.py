@@ -7,7 +7,8 @@ import torch
 
 from oracle import templora_oracle as orc
 from paper_2401_11504_b200 import inputs
-from parity_utils import TOL, assert_close, check_fwd_bwd, f64, hp32, make_state, oracle_fwd_bwd, run_fwd_bwd
+from parity_utils import (TOL, assert_close, check_adam_steps, check_fwd_bwd, f64, hp32, make_state, oracle_fwd_bwd,
+                          run_fwd_bwd, small_gradient_mask)
 
 pytestmark = pytest.mark.gpu
 
@@ -235,10 +236,12 @@ def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True
     assert step == n_steps
     projs = [dict(x=f64(h["x"]), dY=f64(h["dY"]), W0=f64(h["W0"]), s=s, A_master=f64(h["A"]), B_master=f64(h["B"]))
              for h in hosts]
+    grad_log = []
     ref, rstep = orc.update_block(projs, epochs, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"],
                                   bf16_work=(dtype == "bf16"), batch=batch, warmup_steps=warmup,
-                                  lr_round=lambda v: float(np.float32(v)))
+                                  lr_round=lambda v: float(np.float32(v)), grad_log=grad_log)
     assert rstep == step
+    fracs = {}
     epochs = n_steps   # below, "epochs" bounds the number of optimizer steps taken
     tol = TOL[dtype]
     for i, (q, st) in enumerate(zip(ref, states)):
@@ -248,20 +251,16 @@ def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True
         assert_close(f"dA{i}", f64(st["A"]["grad"]), q["dA"], tol)
         assert_close(f"dB{i}", f64(st["B"]["grad"]), q["dB"], tol)
         for nm in ("A", "B"):
-            # master parameters: within tolerance, plus the worst case of the sign-like Adam step on
-            # elements whose gradient is below its own tolerance (2 lr per epoch, see below)
-            err = np.abs(f64(st[nm]["master"]) - q[nm + "_master"]).max()
-            assert err <= tol * np.abs(q[nm + "_master"]).max() + 2.0 * epochs * hp["lr"]
-            # The update itself (|delta| ~ epochs * lr << |p|).  Adam's step is sign-like
-            # (lr * g / (|g| + eps) at step 1), so it is ill-conditioned where |g| is below the
-            # gradient's own tolerance: there the two sides may legitimately differ by up to
-            # 2 lr.  Require agreement everywhere except on a small fraction of such elements.
+            # The update itself (|delta| ~ steps * lr << |p|).  Adam's step is sign-like (lr * g / (|g| + eps) at
+            # step 1), so it is ill-conditioned where |g| is below the gradient's own tolerance: there, and only
+            # there, the two sides may differ, by up to 2 lr per step.  check_adam_steps requires every element
+            # outside the tight bound to be such an element.
             p0 = f64(hosts[i][nm])
-            d_gpu, d_ref = f64(st[nm]["master"]) - p0, q[nm + "_master"] - p0
-            assert np.abs(d_ref).max() > 0
-            bound = tol * np.abs(d_ref).max() + 2.0 ** -23 * np.abs(q[nm + "_master"]).max()
-            outliers = np.abs(d_gpu - d_ref) > bound
-            assert outliers.mean() <= (0.02 if dtype == "bf16" else 1e-3), f"{nm}{i}: {outliers.mean():.4f} of steps off"
+            got = f64(st[nm]["master"])
+            fracs[f"{nm}{i}"] = check_adam_steps(f"{nm}{i}", p0, got, q[nm + "_master"],
+                                                 small_gradient_mask(grad_log, i, nm, tol), tol, epochs, hp["lr"],
+                                                 max_frac=0.02 if dtype == "bf16" else 1e-3)
+            d_gpu = got - p0
             if epochs == 1:
                 # exact check of the optimizer arithmetic: the oracle's step fed with the
                 # gradient the device produced must reproduce the device's step tightly
@@ -274,6 +273,8 @@ def _update_block_case(b, dtype, shapes, T, r, s, epochs, hp, seed, with_dX=True
             assert_close(f"v{nm}{i}", f64(st[nm]["v"]), q["v" + nm], 2 * tol)   # v is quadratic in g
             if dtype == "bf16":
                 assert np.array_equal(f64(st[nm]["work"]), orc.round_bf16(f64(st[nm]["master"]).astype(np.float32)))
+    print("fraction of optimizer steps outside the tight bound (all at gradients within tolerance of zero):",
+          {k: f"{v:.4f}" for k, v in fracs.items()})
 
 
 def test_update_block_fp32_config0(b):

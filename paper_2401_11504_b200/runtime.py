@@ -6,6 +6,8 @@ independent replicas.  The only cross-rank steps are a barrier around the timed 
 over ranks of the measured time, both through torch.distributed (nccl on GPUs, gloo on CPU).
 """
 import os
+import socket
+import subprocess
 import threading
 import time
 
@@ -68,6 +70,49 @@ def aggregate_throughput(units_per_rank, seconds_this_rank, ranks):
     return total_units / slowest, slowest
 
 
+def _free_port():
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_replicas(argv, n, timeout_s=3600):
+    """Start n copies of the command argv as the ranks of one job on this node, one per GPU: RANK and
+    LOCAL_RANK 0..n-1, WORLD_SIZE n, rendezvous on 127.0.0.1 at a free port (what torch.distributed.run
+    would set).  Rank 0's standard output is passed through (it prints the job's one result line); the
+    other ranks' output is dropped, everybody's standard error is passed through.  Returns the first
+    non-zero exit code, or 0.  A rank that fails ends the others: they would wait in the rendezvous for ever."""
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT=str(_free_port()), WORLD_SIZE=str(n))
+    procs = []
+    for rank in range(n):
+        e = dict(env, RANK=str(rank), LOCAL_RANK=str(rank))
+        procs.append(subprocess.Popen(list(argv), env=e, stdout=None if rank == 0 else subprocess.DEVNULL))
+    deadline = time.time() + timeout_s
+    rc = 0
+    pending = list(procs)
+    while pending:
+        for p in list(pending):
+            code = p.poll()
+            if code is None:
+                continue
+            pending.remove(p)
+            if code != 0 and rc == 0:
+                rc = code
+        if rc != 0 or time.time() > deadline:
+            for p in pending:
+                p.terminate()
+            for p in pending:
+                try:
+                    p.wait(timeout=10)
+                except subprocess.TimeoutExpired:
+                    p.kill()
+            if rc == 0:
+                rc = 124
+            break
+        time.sleep(0.05)
+    return rc
+
+
 # ------------------------------------------------------------------ block construction
 class Block:
     """One block of LoRA-augmented projections resident on a device, with optimizer state."""
@@ -127,7 +172,7 @@ class Block:
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
 
-    def __init__(self, cuda_index=0, period_s=0.02):
+    def __init__(self, cuda_index=0, period_s=0.005):
         self.index, self.period = cuda_index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None

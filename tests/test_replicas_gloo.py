@@ -41,6 +41,57 @@ def test_two_replicas_aggregate_over_gloo(tmp_path):
     assert line["slowest"] == 2.0 and abs(line["value"] - 2 * 10240 / 2.0) < 1e-9
 
 
+LAUNCHER = r"""
+import sys
+sys.path.insert(0, sys.argv[1])
+from paper_2401_11504_b200 import runtime
+sys.exit(runtime.spawn_replicas([sys.executable, sys.argv[2], sys.argv[1]] + sys.argv[4:], int(sys.argv[3])))
+"""
+
+
+def _launch(tmp_path, worker_src, n, *extra):
+    worker, launcher = tmp_path / "worker.py", tmp_path / "launcher.py"
+    worker.write_text(worker_src)
+    launcher.write_text(LAUNCHER)
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_PORT")}
+    return subprocess.run([sys.executable, str(launcher), ROOT, str(worker), str(n), *extra], env=env,
+                          capture_output=True, text=True, timeout=300)
+
+
+def test_spawn_replicas_starts_one_rank_per_gpu_and_passes_rank0_output(tmp_path):
+    # what `python bench.py --gpus N` does when it was not started by torch.distributed.run: the same worker as
+    # above, started by runtime.spawn_replicas, which picks the port and sets the rank variables itself
+    res = _launch(tmp_path, WORKER, 2)
+    assert res.returncode == 0, res.stderr[-2000:]
+    import json
+    lines = [l for l in res.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                     # rank 0's line only
+    line = json.loads(lines[0])
+    assert line["slowest"] == 2.0 and abs(line["value"] - 2 * 10240 / 2.0) < 1e-9
+
+
+def test_spawn_replicas_reports_a_failing_rank(tmp_path):
+    # rank 1 exits with an error before the rendezvous: the launcher ends rank 0 (which would wait for ever)
+    # and returns rank 1's code
+    failing = "import os, sys, time\nif os.environ['RANK'] == '1':\n    sys.exit(7)\ntime.sleep(120)\n"
+    res = _launch(tmp_path, failing, 2)
+    assert res.returncode == 7
+
+
+def test_bench_gpus_n_launches_its_own_workers():
+    # without a GPU every worker of `python bench.py --gpus 2` stops at the device check (there is no CPU
+    # path): the run must come back promptly with that error, not with a usage message
+    import pytest
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("this check is for a machine without a GPU")
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "2", "--warmup", "1"],
+                         env=env, capture_output=True, text=True, timeout=600)
+    assert res.returncode != 0
+    assert "needs a CUDA device" in res.stderr and "torch.distributed.run" not in res.stderr
+
+
 def test_single_process_is_world_size_one():
     from paper_2401_11504_b200 import runtime
     env_backup = {k: os.environ.pop(k, None) for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}

@@ -14,6 +14,18 @@ std::atomic<int> g_kernel_path{0};      // 0 = automatic, 1 = generic kernels on
 thread_local int t_path_override = -1;  // set while measuring the workspace needs of both paths
 
 constexpr int kSmRef = 148;  // SM count the split-K heuristic is tuned for (B200)
+#ifndef TL_SPLIT_PER_SM
+#define TL_SPLIT_PER_SM 3
+#endif
+#ifndef TL_SPLIT_MIN_KB
+#define TL_SPLIT_MIN_KB 8
+#endif
+#ifndef TL_ORDER_UV
+#define TL_ORDER_UV 0
+#endif
+#ifndef TL_ORDER_GRADS
+#define TL_ORDER_GRADS 0
+#endif
 
 // Workspace bump allocator.  With base == nullptr it only measures.
 struct WsAlloc {
@@ -39,8 +51,8 @@ inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 // than 8 k-blocks per item, at most 16 splits.
 int pick_splits(int tiles, int kb, int group) {
   long long total = (long long)tiles * kb * (group < 1 ? 1 : group);
-  long long target = (total + kSmRef * 3 - 1) / (kSmRef * 3);
-  if (target < 8) target = 8;
+  long long target = (total + kSmRef * TL_SPLIT_PER_SM - 1) / (kSmRef * TL_SPLIT_PER_SM);
+  if (target < TL_SPLIT_MIN_KB) target = TL_SPLIT_MIN_KB;
   long long s = (kb + target / 2) / target;
   if (s < 1) s = 1;
   if (s > 16) s = 16;
@@ -698,7 +710,7 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
     jobs[nj++] = ReduceJob{b.Upart[i], b.su[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Us[i]};
     jobs[nj++] = ReduceJob{b.Vpart[i], b.sv[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Vs[i]};
   }
-  TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
+  TL_TRY(tc_gemm_grouped(probs, np, 64, status, st, 0, TL_ORDER_UV));
   TL_TRY(reduce_partials_batch(jobs, nj, st));
   // dB and dA go before the frozen-weight GEMMs: they re-read x and dY, which the U, V launch has just
   // pulled through L2 (the big GEMMs stream 1.1 GB and would flush them)
@@ -713,7 +725,7 @@ templora_status_t update_group_tc(const templora_linear_t *proj, const templora_
       if (b.sb[i] > 1) jobs[nj++] = ReduceJob{b.dBpart[i], b.sb[i], nb, nb, 1.f, 1.f, gB, 0, nullptr};
       if (b.sa[i] > 1) jobs[nj++] = ReduceJob{b.dApart[i], b.sa[i], na, na, 1.f, 1.f, gA, 0, nullptr};
     }
-    TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
+    TL_TRY(tc_gemm_grouped(probs, np, 64, status, st, 0, TL_ORDER_GRADS));
     if (nj) TL_TRY(reduce_partials_batch(jobs, nj, st));
     return TEMPLORA_OK;
   };

@@ -180,8 +180,10 @@ struct TcProblem {
 };
 constexpr int kTcMaxProblems = 16;
 // BN: tile width, one of 16, 64, 256.  cta_pairs != 0 with BN == 256 runs 256 x 256 tiles on CTA pairs.
+// order_mode: the order in which the problems' work items are handed out: 0 = heaviest problem first,
+// 1 = as listed, 2 = as listed, backwards.
 templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st,
-                                  int cta_pairs = 0);
+                                  int cta_pairs = 0, int order_mode = 0);
 // Decode-time forward of several projections in one launch: clusters of cluster_size (2 or 4) CTAs split
 // the k-range of each 128-row tile and sum their partial tiles through distributed shared memory.
 // Returns TEMPLORA_ERR_UNSUPPORTED when too few clusters fit (the caller then takes the two-kernel path).

@@ -47,13 +47,23 @@ template <int BN, int STAGES, int TMEM_COLS, int KPS> struct CfgBase {
 };
 template <int BN> struct Cfg;
 template <> struct Cfg<256> : CfgBase<256, 4, 512, 1> {};
-template <> struct Cfg<64> : CfgBase<64, 8, 128, 1> {};
+#ifndef TL_C64_STAGES
+#define TL_C64_STAGES 8
+#endif
+#ifndef TL_C64_KPS
+#define TL_C64_KPS 1
+#endif
+#ifndef TL_C64_HINT
+#define TL_C64_HINT 0
+#endif
+template <> struct Cfg<64> : CfgBase<64, TL_C64_STAGES, 128, TL_C64_KPS> {};
 template <> struct Cfg<16> : CfgBase<16, 3, 32, 4> {};
 
 constexpr int kMaxExtra = 4;   // further operand pairs accumulated into the same output tile
 struct alignas(64) DevProb {
   CUtensorMap tmA, tmB, tmAe, tmBe;
   CUtensorMap tmXa[kMaxExtra], tmXb[kMaxExtra];
+  CUtensorMap tmOut;            // CTA-pair kernel: the bf16 row-major output, boxes of 32 rows x 64 columns
   int kb_x[kMaxExtra], kb_xtot;   // k-blocks of each extra pair and their sum (the pairs follow the extension)
   long long out_s0, out_s1, out_split;
   void *out;
@@ -146,6 +156,27 @@ __device__ __forceinline__ uint64_t l2_policy_evict_first() {
   uint64_t p;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
   return p;
+}
+
+// Bulk tensor store of one box from shared memory (written by this warp through the generic proxy, made
+// visible with fence_proxy_async_smem) to global memory; elements outside the tensor are not written.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// at most N of this thread's bulk groups may still be reading their shared-memory source
+template <int N> __device__ __forceinline__ void bulk_wait_group_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo_f32, uint32_t hi_f32) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(lo_f32), __uint_as_float(hi_f32));
+  return *reinterpret_cast<uint32_t *>(&t);
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -464,7 +495,7 @@ __global__ void __launch_bounds__(kThreads2, 1) tc_gemm_kernel(const __grid_cons
             cur.take(ma, mb, kel);
             const uint32_t sA = smem0 + stage * kStage + j * kSub;
             if (!pa_mn) {
-              if constexpr (BN == 16)   // decode: W0 is read exactly once; keep x, A and the split-K slabs in L2 instead
+              if constexpr (BN == 16 || (BN == 64 && TL_C64_HINT))   // decode: W0 is read exactly once; keep x, A and the split-K slabs in L2 instead
                 tma_load_2d_hint(sA, ma, full_bar(stage), kel, it.m0, stream_policy);
               else
                 tma_load_2d(sA, ma, full_bar(stage), kel, it.m0);
@@ -688,7 +719,13 @@ namespace pair {
 constexpr int kStages = 6;
 constexpr int kStageB = 128 * BK * 2;            // this CTA's half of the B tile: 16 KB
 constexpr int kStage = kStageA + kStageB;        // 32 KB per CTA and stage
-constexpr int kSmemBytes = kStages * kStage + 1024 + 1024;
+// Output staging: each epilogue warp converts its 32 rows x 64 columns of the accumulator to bf16 in a 4 KB
+// buffer (128-byte rows, 128-byte swizzle) and hands it to a bulk tensor store, so that global memory is
+// written in whole 128-byte row segments; two buffers per warp, so the next chunk is converted while the
+// previous one drains.
+constexpr int kOutBox = 32 * 64 * 2;             // 4 KB
+constexpr int kOutStaging = 4 * 2 * kOutBox;     // 32 KB per CTA
+constexpr int kSmemBytes = kStages * kStage + kOutStaging + 1024 + 1024;
 constexpr int kTmemCols = 512;                   // two 256-column accumulators
 constexpr int kPairThreads = 224;                // producer (A), MMA, four epilogue warps, producer (B)
 
@@ -758,18 +795,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_al = smem_raw + (smem0 - smem_u32(smem_raw));
-  const uint32_t bar0 = smem0 + kStages * kStage;
+  const uint32_t out_stage0 = smem0 + kStages * kStage;   // 1024-byte aligned: the swizzle pattern repeats every 1 KB
+  const uint32_t bar0 = out_stage0 + kOutStaging;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };                        // used in the even CTA
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };           // one per CTA
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };       // one per CTA
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };  // used in the even CTA
   const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
-  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + kStages * kStage + 512);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 516);
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + kStages * kStage + kOutStaging + 512);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + kOutStaging + 516);
   // Work items are handed out dynamically: the even CTA's A-operand producer draws them from the counter in
   // the workspace head (heaviest problems come first, so this is longest-processing-time-first scheduling)
   // and writes each into the item rings of both CTAs; every other role takes its items from its CTA's ring.
-  volatile int *sched_ring = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + 528);
+  volatile int *sched_ring = reinterpret_cast<volatile int *>(smem_al + kStages * kStage + kOutStaging + 528);
   const uint32_t ring0 = bar0 + 528;
   auto sfull_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 5 + s); };            // one per CTA
   auto sempty_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 5 + kSched + s); };  // used in the even CTA
@@ -960,6 +998,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     int local = 0, sslot = 0;
     uint32_t sphase = 0;
     bool ok = true;
+    const uint32_t my_stage = out_stage0 + (uint32_t)quarter * (2u * kOutBox);
+    uint32_t chunk_no = 0;   // chunks this warp has staged so far (selects the buffer)
     for (; ok; ++local) {
       int item;
       ok = __all_sync(0xffffffffu, ring_take(sslot, sphase, 610, item));
@@ -975,19 +1015,42 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, g.status, 600)) { ok = false; break; }
       tc_fence_after();
-      const int row = it.m0 + (int)rank * 128 + quarter * 32 + lane;
+      const int row0 = it.m0 + (int)rank * 128 + quarter * 32;   // first of this warp's 32 rows
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 256);
-      uint32_t v[32];
+      uint32_t v[32], w[32];
 #pragma unroll 1
-      for (int c0 = 0; c0 < 256; c0 += 32) {
+      for (int c0 = 0; c0 < 256; c0 += 64, ++chunk_no) {
         tmem_ld32(t_row + c0, v);
+        tmem_ld32(t_row + c0 + 32, w);
+        // the store that read this buffer two chunks ago must be done with it
+        if (lane == 0) bulk_wait_group_read<1>();
         tmem_ld_wait();
-        store_chunk<32>(q, v, row, n0 + c0, 0);
+        __syncwarp();
+        const uint32_t buf = my_stage + (chunk_no & 1u) * (uint32_t)kOutBox;
+        const uint32_t rowp = buf + (uint32_t)lane * 128u;
+        const uint32_t sw = (uint32_t)(lane & 7);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {   // 16-byte piece j of the row holds columns 8j .. 8j+7, stored at piece j ^ (row % 8)
+          st_shared_v4(rowp + (((uint32_t)j ^ sw) << 4), pack_bf16x2(v[8 * j], v[8 * j + 1]),
+                       pack_bf16x2(v[8 * j + 2], v[8 * j + 3]), pack_bf16x2(v[8 * j + 4], v[8 * j + 5]),
+                       pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+          st_shared_v4(rowp + (((uint32_t)(j + 4) ^ sw) << 4), pack_bf16x2(w[8 * j], w[8 * j + 1]),
+                       pack_bf16x2(w[8 * j + 2], w[8 * j + 3]), pack_bf16x2(w[8 * j + 4], w[8 * j + 5]),
+                       pack_bf16x2(w[8 * j + 6], w[8 * j + 7]));
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < q.M && n0 + c0 < q.N) {   // rows and columns beyond the tensor are clipped by the store
+          tma_store_2d(&q.tmOut, buf, n0 + c0, row0);
+          bulk_commit_group();
+        }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
     }
+    if (lane == 0) bulk_wait_group_all();   // every store of this warp has left shared memory and is complete
+    __syncwarp();
   }
 
   tc_fence_before();
@@ -1661,7 +1724,7 @@ bool tc_available() {
 }
 
 templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceStatus *status, cudaStream_t st,
-                                  int cta_pairs) {
+                                  int cta_pairs, int order_mode) {
   if (n <= 0 || n > kTcMaxProblems) return TEMPLORA_ERR_INVALID_ARG;
   const bool use_pair = cta_pairs && BN == 256;   // 256 x 256 tiles on CTA pairs
   const int tile_m = use_pair ? 256 : BM;         // rows of one work item
@@ -1673,7 +1736,7 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
 
   // heaviest work items first: the static round-robin schedule then ends on the short ones
   int order[kTcMaxProblems];
-  for (int i = 0; i < n; ++i) order[i] = i;
+  for (int i = 0; i < n; ++i) order[i] = order_mode == 2 ? n - 1 - i : i;
   auto weight = [&](int i) {
     const TcProblem &p = probs[i];
     long long kb = (p.K + BK - 1) / BK;
@@ -1682,7 +1745,7 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     for (int e = 0; e < p.n_extra; ++e) w += (p.Kx[e] + BK - 1) / BK;
     return w;
   };
-  for (int i = 1; i < n; ++i)
+  for (int i = 1; i < n && order_mode == 0; ++i)
     for (int j = i; j > 0 && weight(order[j]) > weight(order[j - 1]); --j) {
       int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
     }
@@ -1701,7 +1764,9 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     q.kb_main = (p.K + BK - 1) / BK;
     q.kb_ext = (p.Kext + BK - 1) / BK;
     q.splits = p.splits < 1 ? 1 : (p.splits > q.kb_main ? q.kb_main : p.splits);
-    if (use_pair && p.splits > 1) return TEMPLORA_ERR_UNSUPPORTED;
+    if (use_pair && (p.splits > 1 || p.out_f32 || p.out_s1 != 1 || p.epi_mask || (p.out_s0 & 7) ||
+                     (reinterpret_cast<uintptr_t>(p.out) & 15)))
+      return TEMPLORA_ERR_UNSUPPORTED;   // the pair kernel writes bf16 rows through bulk tensor stores
     q.m_tiles = (p.M + tile_m - 1) / tile_m;
     q.n_tiles = (p.N + BN - 1) / BN;
     q.item_start = items;
@@ -1736,9 +1801,12 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
       ok = ok && make_operand_map(&q.tmXa[e], p.Ax[e], p.M, p.Kx[e], p.ldax[e], p.a_mn, BM) &&
            make_operand_map(&q.tmXb[e], p.Bx[e], p.N, p.Kx[e], p.ldbx[e], p.b_mn, box_b);
     }
+    if (use_pair) ok = ok && make_map(&q.tmOut, p.out, p.N, p.M, p.out_s0, 32);
+    else q.tmOut = q.tmA;
     if (!ok) return TEMPLORA_ERR_CUDA;
   }
   g.n_items = items;
+  static_assert(sizeof(DevGroup) <= 32000, "the launch description travels as a kernel parameter");
   if (use_pair) return launch_pair(g, di, st);
   if (BN == 256) return launch<256>(g, di, 0, st);
   if (BN == 64) return launch<64>(g, di, 1, st);
@@ -1779,6 +1847,7 @@ templora_status_t tc_decode_cluster(const TcProblem *probs, int n, int n_tokens,
     q.pad = p.role; q.pad3 = p.flag;
     q.kb_xtot = 0;
     for (int e = 0; e < kMaxExtra; ++e) { q.kb_x[e] = 0; q.tmXa[e] = q.tmA; q.tmXb[e] = q.tmB; }
+    q.tmOut = q.tmA;
     q.epi_mask = nullptr; q.epi_mask_pitch = 0; q.epi_scale = p.epi_scale;
     q.out = p.out; q.out_s0 = 1; q.out_s1 = p.out_s1; q.out_split = 0;
     items += q.m_tiles;

@@ -1090,6 +1090,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 // counter and writes them into every CTA's item ring.
 namespace dcl {
 
+#ifndef TL_DCL_EARLY
+#define TL_DCL_EARLY 1
+#endif
+
 constexpr int kSub = kStageA + 16 * BK * 2;        // one k-block: 128 x 64 of W0 + 16 x 64 of x
 // Shared memory of a CTA: the operand ring (n_stages stages of KPS k-blocks), then room for the partial
 // tiles of the S - 1 other CTAs (used in CTA 0 only, but every CTA of a launch has the same layout;
@@ -1186,7 +1190,12 @@ __global__ void __launch_bounds__(kThreads, 1)
   pair::cluster_sync_all();   // the peers' barriers are initialised before anything is sent to them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_prologue();
+  // Ordering against the kernels ahead on the stream.  Everything this kernel reads may have been written by them
+  // EXCEPT the frozen weights W0, which nothing ever writes: the producer thread requests the W0 tiles of its
+  // cluster's first item before it waits for the predecessors (the requests then overlap the predecessor's last
+  // items and the completion hand-over between the two grids), every other thread waits here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!(TL_DCL_EARLY && warp == 0)) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // this CTA's share of an item.  The streamed operand's k-blocks are dealt to the S CTAs in chunks of KPS
   // (one pipeline stage) round-robin, so at any time the cluster reads neighbouring pieces of the same
@@ -1235,6 +1244,38 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
         return true;
       };
+      // The cluster's first item is known without the counter (cluster c starts on item c).  When it is a y item,
+      // the W0 part of its first stages is requested now, the x part right after the wait below.
+      int pre_chunks = 0;
+      if (TL_DCL_EARLY) {
+        if (item < g.n_items) {
+          int p, m0, nmain, next;
+          share_of(item, p, m0, nmain, next);
+          const DevProb &q = g.p[p];
+          if (q.pad == 0) {   // role 0: the streamed operand is W0
+            pre_chunks = nmain / kKps;   // whole stages made of streamed k-blocks only
+            if (pre_chunks > kStages) pre_chunks = kStages;
+            for (int c = 0; c < pre_chunks; ++c) {
+              mbar_arrive_expect_tx(full_bar(c), (uint32_t)(kKps * kSub));
+              for (int j = 0; j < kKps; ++j) {
+                const int kel = ((c * S + rank) * kKps + j) * BK;
+                tma_load_2d_hint(smem0 + c * kStage + j * kSub, &q.tmA, full_bar(c), kel, m0, stream_policy);
+              }
+            }
+          }
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (pre_chunks) {
+          int p, m0, nmain, next;
+          share_of(item, p, m0, nmain, next);
+          const DevProb &q = g.p[p];
+          for (int c = 0; c < pre_chunks; ++c)
+            for (int j = 0; j < kKps; ++j) {
+              const int kel = ((c * S + rank) * kKps + j) * BK;
+              tma_load_2d(smem0 + c * kStage + j * kSub + kStageA, &q.tmB, full_bar(c), kel, 0);
+            }
+        }
+      }
       // CTA 0 deals one item ahead (the peers learn the next item before this CTA starts loading the
       // current one) and draws two ahead, so the counter's round trip is never waited for
       int next_item = 0, drawn = 0;
@@ -1262,6 +1303,12 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (!u_ready) { f0 = ld_volatile_i4(flags); f1 = ld_volatile_i4(flags + 4); }
         for (int i0 = 0; ok && i0 < nkb; i0 += kKps) {
           const int cnt = (nkb - i0 < kKps) ? nkb - i0 : kKps;
+          if (pre_chunks > 0) {   // this stage of the first item was requested before the loop
+            --pre_chunks;
+            ++issued;
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           if (!u_ready && i0 + cnt > nmain) {
             // s*u of this projection must be complete (another cluster writes it): bounded wait on its flag.
             // One pass reads the flags of all projections, so each is usually waited for once per CTA.

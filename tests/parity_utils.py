@@ -38,6 +38,43 @@ def f64(t):
     return inputs.to_f64(t)
 
 
+class Guarded:
+    """Device buffers with canary words on both sides.  compute-sanitizer is not available where these tests run,
+    so writes past the ends of an output or of the workspace are caught this way: every buffer handed to the
+    library sits inside a larger allocation whose margins hold a fixed bit pattern, and check() requires the
+    margins to be bit-for-bit intact afterwards.  (NaN-filled outputs show elements that were NOT written; the
+    margins show writes that should not have happened.)"""
+    MARGIN = 4096          # bytes on each side; a multiple of 1024 so that a workspace keeps its alignment
+    PATTERN = 0xA5
+
+    def __init__(self):
+        self.items = []
+
+    def empty(self, shape, dtype, fill=float("nan")):
+        n = int(np.prod(shape))
+        esize = torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((2 * self.MARGIN + n * esize,), self.PATTERN, dtype=torch.uint8, device="cuda")
+        view = raw[self.MARGIN:self.MARGIN + n * esize].view(dtype).view(*shape)
+        view.fill_(fill)
+        self.items.append((raw, n * esize))
+        return view
+
+    def workspace(self, nbytes):
+        nbytes = int(nbytes)
+        raw = torch.full((2 * self.MARGIN + nbytes,), self.PATTERN, dtype=torch.uint8, device="cuda")
+        view = raw[self.MARGIN:self.MARGIN + nbytes]
+        view.zero_()
+        assert view.data_ptr() % 256 == 0
+        self.items.append((raw, nbytes))
+        return view
+
+    def check(self, what=""):
+        for k, (raw, nbytes) in enumerate(self.items):
+            lo, hi = raw[:self.MARGIN], raw[self.MARGIN + nbytes:]
+            assert bool((lo == self.PATTERN).all()), f"{what}: buffer {k}: bytes BEFORE its start were overwritten"
+            assert bool((hi == self.PATTERN).all()), f"{what}: buffer {k}: bytes PAST its end were overwritten"
+
+
 def run_fwd_bwd(b, host, s, T, with_dX=True, save_U=True, accumulate=False, dropout=None):
     """host: dict of CPU tensors (x, W0, A, B, dY).  Returns GPU outputs as float64 numpy."""
     dev = {k: v.cuda() for k, v in host.items()}
@@ -45,16 +82,19 @@ def run_fwd_bwd(b, host, s, T, with_dX=True, save_U=True, accumulate=False, drop
     r = host["A"].shape[0]
     dkw = {} if dropout is None else dict(dropout_p=dropout[0], dropout_seed=dropout[1], dropout_offset=dropout[2])
     lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], s, **dkw)
-    ws = b.alloc_workspace(b.templora_workspace_bytes(lin, T))
+    guard = Guarded()       # every output and the workspace carry canary margins
+    ws = guard.workspace(b.templora_workspace_bytes(lin, T))
     dt = host["x"].dtype
-    y = torch.full((T, d_out), float("nan"), dtype=dt, device="cuda")
-    dX = torch.full((T, d_in), float("nan"), dtype=dt, device="cuda") if with_dX else None
-    U = torch.full((T, r), float("nan"), dtype=torch.float32, device="cuda") if save_U else None
+    y = guard.empty((T, d_out), dt)
+    dX = guard.empty((T, d_in), dt) if with_dX else None
+    U = guard.empty((T, r), torch.float32) if save_U else None
     init = 1.0 if accumulate else float("nan")
-    dA = torch.full((r, d_in), init, dtype=torch.float32, device="cuda")
-    dB = torch.full((d_out, r), init, dtype=torch.float32, device="cuda")
+    dA = guard.empty((r, d_in), torch.float32, init)
+    dB = guard.empty((d_out, r), torch.float32, init)
     b.templora_linear_fwd(lin, dev["x"], y, ws, U_save=U)
+    guard.check("after templora_linear_fwd")
     b.templora_linear_bwd(lin, dev["x"], dev["dY"], dX, dA, dB, ws, U_saved=U, accumulate=accumulate)
+    guard.check("after templora_linear_bwd")
     code, where = b.templora_read_device_status(ws)
     assert code == 0, f"device status {code} at {where}"
     out = dict(y=f64(y), dA=f64(dA), dB=f64(dB))

@@ -7,7 +7,7 @@ import torch
 
 from oracle import templora_oracle as orc
 from paper_2401_11504_b200 import inputs
-from parity_utils import (TOL, assert_close, check_adam_steps, check_fwd_bwd, f64, hp32, make_state, oracle_fwd_bwd,
+from parity_utils import (TOL, Guarded, assert_close, check_adam_steps, check_fwd_bwd, f64, hp32, make_state, oracle_fwd_bwd,
                           run_fwd_bwd, ill_conditioned_mask)
 
 pytestmark = pytest.mark.gpu
@@ -97,10 +97,12 @@ def test_decode_matches_oracle(b, n, d_in, d_out, r):
     host = inputs.make_linear(9, f"dec-{n}-{d_in}-{d_out}", n, d_in, d_out, r, dtype="bf16")
     dev = {k: v.cuda() for k, v in host.items()}
     lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], 2.0)
-    ws = b.alloc_workspace(b.templora_workspace_bytes(lin, 16))
-    y = torch.full((n, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+    guard = Guarded()
+    ws = guard.workspace(b.templora_workspace_bytes(lin, 16))
+    y = guard.empty((n, d_out), torch.bfloat16)
     b.templora_decode_fwd(lin, dev["x"], y, ws)
     assert b.templora_read_device_status(ws)[0] == 0
+    guard.check("after templora_decode_fwd")
     ref = orc.decode_fwd(f64(host["x"]), f64(host["W0"]), f64(host["A"]), f64(host["B"]), 2.0)
     assert_close("decode y", f64(y), ref, TOL["bf16"])
 
@@ -126,11 +128,13 @@ def test_decode_block_matches_oracle(b):
         hosts = [inputs.make_linear(14, f"decblk-{n}-{i}", n, di, do, r, dtype="bf16") for i, (di, do, r) in enumerate(shapes)]
         devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
         lins = [b.linear_desc(d["W0"], d["A"], d["B"], 2.0) for d in devs]
-        ys = [torch.full((n, do), float("nan"), dtype=torch.bfloat16, device="cuda") for _, do, _ in shapes]
-        ws = b.alloc_workspace(b.templora_decode_block_workspace_bytes(lins))
+        guard = Guarded()
+        ys = [guard.empty((n, do), torch.bfloat16) for _, do, _ in shapes]
+        ws = guard.workspace(b.templora_decode_block_workspace_bytes(lins))
         args = b.DecodeBlockArgs(lins, [d["x"] for d in devs], ys)
         b.templora_decode_block_fwd(args, ws)
         assert b.templora_read_device_status(ws)[0] == 0
+        guard.check(f"after templora_decode_block_fwd n={n}")
         for i, h in enumerate(hosts):
             ref = orc.decode_fwd(f64(h["x"]), f64(h["W0"]), f64(h["A"]), f64(h["B"]), 2.0)
             assert_close(f"decode block y{i} n={n}", f64(ys[i]), ref, TOL["bf16"])
@@ -421,11 +425,13 @@ def _decode_case(b, seed, tag, n, d_in, d_out, r, ws=None):
     host = inputs.make_linear(seed, tag, n, d_in, d_out, r, dtype="bf16")
     dev = {k: v.cuda() for k, v in host.items()}
     lin = b.linear_desc(dev["W0"], dev["A"], dev["B"], 2.0)
+    guard = Guarded()
     if ws is None:
-        ws = b.alloc_workspace(b.templora_workspace_bytes(lin, 16))
-    y = torch.full((n, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+        ws = guard.workspace(b.templora_workspace_bytes(lin, 16))
+    y = guard.empty((n, d_out), torch.bfloat16)
     b.templora_decode_fwd(lin, dev["x"], y, ws)
     assert b.templora_read_device_status(ws)[0] == 0
+    guard.check(f"after templora_decode_fwd ({tag})")
     ref = orc.decode_fwd(f64(host["x"]), f64(host["W0"]), f64(host["A"]), f64(host["B"]), 2.0)
     assert_close(f"decode y {tag}", f64(y), ref, TOL["bf16"])
     return ws

@@ -251,6 +251,29 @@ templora_status_t templora_rmsnorm_bwd(int32_t T, int32_t d, int32_t dtype, cons
                                        float eps, void *dx, void *stream);
 
 /*
+ * The chunk update of the MLP of a Llama-style decoder block in one call ("Train Theta_k", Algorithm 1, run over
+ * the block's gate, up and down projections with the gating between them; the gating is the model's, see above):
+ *     gate = x Wg^T + s (x Ag^T) Bg^T     up = x Wu^T + s (x Au^T) Bu^T     h = SiLU(gate) * up
+ *     y    = h Wd^T + s (h Ad^T) Bd^T
+ * and, from dY (the gradient with respect to y), the backward through down, the gating and gate/up:
+ *     dh = dY Wd + s (dY Bd) Ad;  dgate, dup as in templora_swiglu_bwd;
+ *     dX = dgate Wg + dup Wu + s (dgate Bg) Ag + s (dup Bu) Au      (the gradient with respect to x)
+ * with the six LoRA gradients as in templora_linear_bwd, then one AdamW step on all six tensors; `epochs` times.
+ *   proj, A_state, B_state: HOST arrays of three entries in the order gate, up, down, aliased as in
+ *   templora_update_block; gate.d_in == up.d_in, gate.d_out == up.d_out == down.d_in; dropout_p must be 0.
+ *   x [T, d_in], dY [T, down.d_out] inputs; gate, up, h [T, d_ff] and y [T, down.d_out] outputs (gate and up are the
+ *   pre-activations the backward reads); dX [T, d_in] output or NULL.  All device buffers of the projections' dtype.
+ * On the tensor-core path the gating costs no pass of its own: gate and up are one GEMM whose epilogue also
+ * writes h, and dh is never stored: the epilogue of the down projection's input gradient writes dgate and dup.
+ */
+size_t templora_update_mlp_workspace_bytes(const templora_linear_t *proj, int32_t T);
+templora_status_t templora_update_mlp(const templora_linear_t *proj, const templora_param_t *A_state,
+                                      const templora_param_t *B_state, int32_t T, const void *x, const void *dY,
+                                      void *gate, void *up, void *h, void *y, void *dX, int32_t epochs, float lr,
+                                      float beta1, float beta2, float eps, float weight_decay, int64_t *step_inout,
+                                      void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Failure-detection self-test (the paper has no counterpart).  Enqueues one tiny kernel that
  * waits, the way the GEMM kernels wait for their copies, on a barrier that nothing signals.
  * After limit_ms (1..1000) it records TEMPLORA_ERR_TIMEOUT in the status record at the head of

@@ -24,7 +24,8 @@ EXPORTS = [
     "templora_decode_block_workspace_bytes", "templora_decode_block_fwd", "templora_update_block_batched",
     "templora_set_stream_sm_limit", "templora_selftest_bounded_wait", "templora_lr_at_step",
     "templora_update_block_warmup", "templora_swiglu_fwd", "templora_swiglu_bwd", "templora_rmsnorm_fwd",
-    "templora_rmsnorm_bwd", "templora_decode_fwd_noalloc_status",
+    "templora_rmsnorm_bwd", "templora_decode_fwd_noalloc_status", "templora_update_mlp",
+    "templora_update_mlp_workspace_bytes",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 (KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
@@ -78,6 +79,11 @@ def _load():
     lib.templora_update_block_warmup.restype = i32
     lib.templora_update_block_warmup.argtypes = [LP, PP, PP, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                                  C.POINTER(vp), i32, f32, i64, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
+    lib.templora_update_mlp_workspace_bytes.restype = sz
+    lib.templora_update_mlp_workspace_bytes.argtypes = [LP, i32]
+    lib.templora_update_mlp.restype = i32
+    lib.templora_update_mlp.argtypes = [LP, PP, PP, i32, vp, vp, vp, vp, vp, vp, vp, i32, f32, f32, f32, f32, f32,
+                                        C.POINTER(i64), vp, sz, vp]
     lib.templora_swiglu_fwd.restype = i32
     lib.templora_swiglu_fwd.argtypes = [i64, i32, vp, vp, vp, vp]
     lib.templora_swiglu_bwd.restype = i32
@@ -249,6 +255,22 @@ def templora_update_block_warmup(args, batch_tokens, epochs, lr, warmup_steps, b
                                             args.dY, args.y, args.dX, int(epochs), lr, int(warmup_steps), beta1, beta2,
                                             eps, weight_decay, C.byref(st), _ptr(ws), ws.numel(), _stream(stream)),
            "templora_update_block_warmup")
+    return st.value
+
+
+def templora_update_mlp_workspace_bytes(lins, T):
+    arr = (LinearDesc * 3)(*lins)
+    return int(lib.templora_update_mlp_workspace_bytes(arr, int(T)))
+
+
+def templora_update_mlp(lins, A_states, B_states, x, dY, gate, up, h, y, dX, epochs, lr, beta1, beta2, eps, weight_decay,
+                        step, ws, stream=None):
+    """Chunk update of a block's MLP (lins, A_states, B_states: gate, up, down); returns the new step count."""
+    st = C.c_int64(int(step))
+    _check(lib.templora_update_mlp((LinearDesc * 3)(*lins), (ParamDesc * 3)(*A_states), (ParamDesc * 3)(*B_states),
+                                   x.shape[0], _ptr(x), _ptr(dY), _ptr(gate), _ptr(up), _ptr(h), _ptr(y), _ptr(dX),
+                                   int(epochs), lr, beta1, beta2, eps, weight_decay, C.byref(st), _ptr(ws), ws.numel(),
+                                   _stream(stream)), "templora_update_mlp")
     return st.value
 
 

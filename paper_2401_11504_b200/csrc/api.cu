@@ -870,6 +870,179 @@ templora_status_t update_impl(const templora_linear_t *proj, const templora_para
   return TEMPLORA_OK;
 }
 
+
+// ---------------------------------------------------------------- the MLP of a decoder block in one call
+// gate = x Wg^T + s (x Ag^T) Bg^T,  up likewise,  h = SiLU(gate) * up,  y = h Wd^T + s (h Ad^T) Bd^T;
+// backward from dY through down, the gating and gate/up to dX (the gradient with respect to x, the sum of the
+// gate and up branches) and the six LoRA gradients; AdamW on all six.  proj = {gate, up, down}.
+// On the tensor-core path with CTA pairs the gating runs in the epilogues of the frozen-weight GEMMs: gate and up
+// are ONE problem whose tiles hold 128 columns of each and whose epilogue writes gate, up and h; the down
+// projection's input gradient dh is never stored, its epilogue writes dgate and dup.
+templora_status_t mlp_impl(const templora_linear_t *proj, const templora_param_t *As, const templora_param_t *Bs, int T,
+                           const void *x, const void *dY, void *gate, void *up, void *h, void *y, void *dX, int epochs,
+                           float lr, float b1, float b2, float eps, float wd, int64_t *step_inout, void *ws_ptr,
+                           size_t ws_bytes, bool dry, size_t *need, cudaStream_t st) {
+  const templora_linear_t *lg = proj, *lu = proj + 1, *ld = proj + 2;
+  const int d_ff = lg->d_out;
+  const size_t esize = lg->dtype == TEMPLORA_BF16 ? 2 : 4;
+  const bool all_tc = use_tc(lg, dry) && use_tc(lu, dry) && use_tc(ld, dry);
+  const bool fused = all_tc && use_pairs() && lg->r == lu->r;
+  const int work_bf16 = lg->dtype == TEMPLORA_BF16;
+  std::vector<templora_param_t> all;
+  if (!dry)
+    for (int i = 0; i < 3; ++i) { all.push_back(As[i]); all.push_back(Bs[i]); }
+  int64_t step = dry ? 0 : *step_inout;
+
+  if (all_tc) {
+    WsAlloc a(dry ? nullptr : ws_ptr, ws_bytes);
+    GroupBufs b;
+    carve_group(proj, 3, T, a, b);
+    __nv_bfloat16 *dgate = a.take<__nv_bfloat16>((size_t)T * d_ff);
+    __nv_bfloat16 *dup = a.take<__nv_bfloat16>((size_t)T * d_ff);
+    __nv_bfloat16 *dh = a.take<__nv_bfloat16>((size_t)T * d_ff);   // used only when the gating is not fused
+    if (need) *need = a.off;
+    if (dry) return TEMPLORA_OK;
+    if (a.overflow) return TEMPLORA_ERR_WORKSPACE;
+    DeviceStatus *status = a.status();
+    auto reduce_uv = [&](int i, bool u, bool v) -> templora_status_t {
+      ReduceJob jobs[2];
+      int nj = 0;
+      const long long Tr = (long long)T * proj[i].r;
+      if (u) jobs[nj++] = ReduceJob{b.Upart[i], b.su[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Us[i]};
+      if (v) jobs[nj++] = ReduceJob{b.Vpart[i], b.sv[i], Tr, Tr, proj[i].s, 1.f, nullptr, 0, b.Vs[i]};
+      return reduce_partials_batch(jobs, nj, st);
+    };
+    auto grads = [&](const int *which, int n, const void *const *xin, const void *const *dyin) -> templora_status_t {
+      TcProblem probs[4];
+      ReduceJob jobs[4];
+      int np = 0, nj = 0;
+      for (int k = 0; k < n; ++k) {
+        const int i = which[k];
+        const templora_linear_t *l = proj + i;
+        float *gB = const_cast<float *>(Bs[i].grad), *gA = const_cast<float *>(As[i].grad);
+        probs[np++] = prob_dB(l, T, dyin[k], b.Us[i], b.sb[i] > 1 ? b.dBpart[i] : gB, b.sb[i]);
+        probs[np++] = prob_dA(l, T, xin[k], b.Vs[i], b.sa[i] > 1 ? b.dApart[i] : gA, b.sa[i]);
+        const long long nb = (long long)l->d_out * l->r, na = (long long)l->d_in * l->r;
+        if (b.sb[i] > 1) jobs[nj++] = ReduceJob{b.dBpart[i], b.sb[i], nb, nb, 1.f, 1.f, gB, 0, nullptr};
+        if (b.sa[i] > 1) jobs[nj++] = ReduceJob{b.dApart[i], b.sa[i], na, na, 1.f, 1.f, gA, 0, nullptr};
+      }
+      TL_TRY(tc_gemm_grouped(probs, np, 64, status, st));
+      if (nj) TL_TRY(reduce_partials_batch(jobs, nj, st));
+      return TEMPLORA_OK;
+    };
+    for (int e = 0; e < epochs; ++e) {
+      // forward: U of gate and up, then gate | up | h in one launch
+      TcProblem sk[2] = {prob_U(lg, T, x, b.Upart[0], b.su[0]), prob_U(lu, T, x, b.Upart[1], b.su[1])};
+      TL_TRY(tc_gemm_grouped(sk, 2, 64, status, st));
+      {
+        const long long Tr0 = (long long)T * lg->r, Tr1 = (long long)T * lu->r;
+        ReduceJob jobs[2] = {ReduceJob{b.Upart[0], b.su[0], Tr0, Tr0, lg->s, 1.f, nullptr, 0, b.Us[0]},
+                             ReduceJob{b.Upart[1], b.su[1], Tr1, Tr1, lu->s, 1.f, nullptr, 0, b.Us[1]}};
+        TL_TRY(reduce_partials_batch(jobs, 2, st));
+      }
+      if (fused) {
+        TcProblem p = prob_y(lg, T, x, b.Us[0], gate);
+        p.epi_mode = 1;
+        p.B1 = lu->W0; p.ldb1 = lu->d_in;
+        p.Bext1 = lu->B; p.ldbext1 = lu->r;
+        p.Aext1 = b.Us[1]; p.ldaext1 = lu->r;
+        p.out1 = up; p.out2 = h;
+        TL_TRY(tc_gemm_grouped(&p, 1, 256, status, st, 1));
+      } else {
+        TcProblem p[2] = {prob_y(lg, T, x, b.Us[0], gate), prob_y(lu, T, x, b.Us[1], up)};
+        TL_TRY(tc_gemm_grouped(p, 2, 256, status, st, use_pairs()));
+        TL_TRY(templora_swiglu_fwd((int64_t)T * d_ff, lg->dtype, gate, up, h, st));
+      }
+      // down: U from h, V from dY; its LoRA gradients; y and the gradient with respect to h
+      sk[0] = prob_U(ld, T, h, b.Upart[2], b.su[2]);
+      sk[1] = prob_V(ld, T, dY, b.Vpart[2], b.sv[2]);
+      TL_TRY(tc_gemm_grouped(sk, 2, 64, status, st));
+      TL_TRY(reduce_uv(2, true, true));
+      {
+        const int which[1] = {2};
+        const void *xin[1] = {h}, *dyin[1] = {dY};
+        TL_TRY(grads(which, 1, xin, dyin));
+      }
+      {
+        TcProblem p[2] = {prob_y(ld, T, h, b.Us[2], y), prob_dX(ld, T, dY, b.Vs[2], fused ? dgate : dh)};
+        if (fused) {
+          p[1].epi_mode = 2;
+          p[1].out1 = dup;
+          p[1].epi_in0 = gate; p[1].epi_in1 = up;
+        }
+        TL_TRY(tc_gemm_grouped(p, 2, 256, status, st, use_pairs()));
+        if (!fused) TL_TRY(templora_swiglu_bwd((int64_t)T * d_ff, lg->dtype, gate, up, dh, dgate, dup, st));
+      }
+      // gate and up backward: V, the LoRA gradients, and one summed input gradient
+      sk[0] = prob_V(lg, T, dgate, b.Vpart[0], b.sv[0]);
+      sk[1] = prob_V(lu, T, dup, b.Vpart[1], b.sv[1]);
+      TL_TRY(tc_gemm_grouped(sk, 2, 64, status, st));
+      {
+        const long long Tr0 = (long long)T * lg->r, Tr1 = (long long)T * lu->r;
+        ReduceJob jobs[2] = {ReduceJob{b.Vpart[0], b.sv[0], Tr0, Tr0, lg->s, 1.f, nullptr, 0, b.Vs[0]},
+                             ReduceJob{b.Vpart[1], b.sv[1], Tr1, Tr1, lu->s, 1.f, nullptr, 0, b.Vs[1]}};
+        TL_TRY(reduce_partials_batch(jobs, 2, st));
+      }
+      {
+        const int which[2] = {0, 1};
+        const void *xin[2] = {x, x}, *dyin[2] = {dgate, dup};
+        TL_TRY(grads(which, 2, xin, dyin));
+      }
+      if (dX) {
+        TcProblem p = prob_dX(lg, T, dgate, b.Vs[0], dX);
+        p.n_extra = 2;
+        p.Ax[0] = dup; p.ldax[0] = d_ff; p.Bx[0] = lu->W0; p.ldbx[0] = lu->d_in; p.Kx[0] = d_ff;
+        p.Ax[1] = b.Vs[1]; p.ldax[1] = lu->r; p.Bx[1] = lu->A; p.ldbx[1] = lu->d_in; p.Kx[1] = lu->r;
+        TL_TRY(tc_gemm_grouped(&p, 1, 256, status, st, use_pairs()));
+      }
+      ++step;
+      TL_TRY(adamw_launch(all.data(), 6, lr, b1, b2, eps, wd, step, work_bf16, st));
+      *step_inout = step;
+    }
+    return TEMPLORA_OK;
+  }
+
+  // generic kernels: the same chain from the single-projection pieces
+  const int saved_override = t_path_override;
+  t_path_override = 1;
+  auto restore = [&](templora_status_t rc) { t_path_override = saved_override; return rc; };
+  WsAlloc a(dry ? nullptr : ws_ptr, ws_bytes);
+  uint8_t *dgate = a.take<uint8_t>((size_t)T * d_ff * esize);
+  uint8_t *dup = a.take<uint8_t>((size_t)T * d_ff * esize);
+  uint8_t *dh = a.take<uint8_t>((size_t)T * d_ff * esize);
+  size_t max_need = a.off;
+  for (int i = 0; i < 3; ++i) {
+    WsAlloc m = a, m2 = a;
+    fwd_impl(proj + i, T, nullptr, nullptr, nullptr, m, true, st);
+    bwd_impl(proj + i, T, nullptr, nullptr, nullptr, reinterpret_cast<void *>(16), nullptr, nullptr, 0, m2, true, st, 1);
+    if (m.off > max_need) max_need = m.off;
+    if (m2.off > max_need) max_need = m2.off;
+  }
+  if (need) *need = max_need;
+  if (dry) return restore(TEMPLORA_OK);
+  if (ws_bytes < max_need) return restore(TEMPLORA_ERR_WORKSPACE);
+  for (int e = 0; e < epochs; ++e) {
+    auto run = [&]() -> templora_status_t {
+      { WsAlloc c = a; TL_TRY(fwd_impl(lg, T, x, gate, nullptr, c, false, st)); }
+      { WsAlloc c = a; TL_TRY(fwd_impl(lu, T, x, up, nullptr, c, false, st)); }
+      TL_TRY(templora_swiglu_fwd((int64_t)T * d_ff, lg->dtype, gate, up, h, st));
+      { WsAlloc c = a; TL_TRY(fwd_impl(ld, T, h, y, nullptr, c, false, st)); }
+      { WsAlloc c = a; TL_TRY(bwd_impl(ld, T, h, dY, nullptr, dh, const_cast<float *>(As[2].grad), const_cast<float *>(Bs[2].grad), 0, c, false, st)); }
+      TL_TRY(templora_swiglu_bwd((int64_t)T * d_ff, lg->dtype, gate, up, dh, dgate, dup, st));
+      { WsAlloc c = a; TL_TRY(bwd_impl(lg, T, x, dgate, nullptr, dX, const_cast<float *>(As[0].grad), const_cast<float *>(Bs[0].grad), 0, c, false, st)); }
+      { WsAlloc c = a; TL_TRY(bwd_impl(lu, T, x, dup, nullptr, dX, const_cast<float *>(As[1].grad), const_cast<float *>(Bs[1].grad), 0, c, false, st, dX ? 1 : 0)); }
+      return TEMPLORA_OK;
+    };
+    const templora_status_t rc = run();
+    if (rc != TEMPLORA_OK) return restore(rc);
+    ++step;
+    const templora_status_t ra = adamw_launch(all.data(), 6, lr, b1, b2, eps, wd, step, work_bf16, st);
+    if (ra != TEMPLORA_OK) return restore(ra);
+    *step_inout = step;
+  }
+  return restore(TEMPLORA_OK);
+}
+
 }  // namespace
 
 // Workspace bytes that templora_decode_fwd alone needs for n tokens (0 on an invalid projection);
@@ -1084,6 +1257,63 @@ templora_status_t templora_update_block_warmup(const templora_linear_t *proj, co
   return update_impl(proj, A_state, B_state, n_proj, T, batch_tokens, x, dY, y, dX, epochs, lr, beta1, beta2, eps,
                      weight_decay, step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream),
                      warmup_steps);
+}
+
+static templora_status_t check_mlp(const templora_linear_t *proj) {
+  if (!proj) return TEMPLORA_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i) {
+    TL_TRY(check_linear(proj + i));
+    if (proj[i].dtype != proj[0].dtype) return TEMPLORA_ERR_UNSUPPORTED;
+    if (proj[i].dropout_p != 0.f) return TEMPLORA_ERR_UNSUPPORTED;
+  }
+  // gate and up read the same input and feed the gating; down reads its result
+  if (proj[0].d_in != proj[1].d_in || proj[0].d_out != proj[1].d_out || proj[2].d_in != proj[0].d_out)
+    return TEMPLORA_ERR_INVALID_ARG;
+  return TEMPLORA_OK;
+}
+
+size_t templora_update_mlp_workspace_bytes(const templora_linear_t *proj, int32_t T) {
+  if (check_mlp(proj) != TEMPLORA_OK || T <= 0) return 0;
+  size_t need = 0, best = kStatusBytes;
+  for (int mode = 0; mode < 2; ++mode) {
+    t_path_override = mode;
+    mlp_impl(proj, nullptr, nullptr, T, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0, 0,
+             nullptr, nullptr, 0, true, &need, nullptr);
+    if (need > best) best = need;
+  }
+  t_path_override = -1;
+  return best;
+}
+
+templora_status_t templora_update_mlp(const templora_linear_t *proj, const templora_param_t *A_state,
+                                      const templora_param_t *B_state, int32_t T, const void *x, const void *dY,
+                                      void *gate, void *up, void *h, void *y, void *dX, int32_t epochs, float lr,
+                                      float beta1, float beta2, float eps, float weight_decay, int64_t *step_inout,
+                                      void *ws, size_t ws_bytes, void *stream) {
+  TL_TRY(check_mlp(proj));
+  if (!A_state || !B_state || T <= 0 || !x || !dY || !gate || !up || !h || !y || epochs < 0 || !step_inout || *step_inout < 0)
+    return TEMPLORA_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f)) return TEMPLORA_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(dY) || !aligned16(gate) || !aligned16(up) || !aligned16(h) || !aligned16(y) ||
+      (dX && !aligned16(dX)))
+    return TEMPLORA_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i) {
+    TL_TRY(check_linear_ptrs(proj + i));
+    const templora_param_t &a = A_state[i], &b = B_state[i];
+    if (a.n != (int64_t)proj[i].r * proj[i].d_in || b.n != (int64_t)proj[i].d_out * proj[i].r) return TEMPLORA_ERR_INVALID_ARG;
+    if (!a.master || !a.m || !a.v || !a.grad || !b.master || !b.m || !b.v || !b.grad) return TEMPLORA_ERR_INVALID_ARG;
+    if (!aligned16(a.grad) || !aligned16(b.grad)) return TEMPLORA_ERR_INVALID_ARG;
+    const void *wa = proj[i].dtype == TEMPLORA_BF16 ? a.work : (const void *)a.master;
+    const void *wb = proj[i].dtype == TEMPLORA_BF16 ? b.work : (const void *)b.master;
+    if (proj[i].A != wa || proj[i].B != wb) return TEMPLORA_ERR_INVALID_ARG;
+  }
+  TL_TRY(check_ws(ws, ws_bytes));
+  size_t need = 0;
+  mlp_impl(proj, nullptr, nullptr, T, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0, 0, nullptr,
+           nullptr, 0, true, &need, nullptr);
+  if (ws_bytes < need) return TEMPLORA_ERR_WORKSPACE;
+  return mlp_impl(proj, A_state, B_state, T, x, dY, gate, up, h, y, dX, epochs, lr, beta1, beta2, eps, weight_decay,
+                  step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream));
 }
 
 const char *templora_status_string(templora_status_t st) {

@@ -174,6 +174,19 @@ struct TcProblem {
   const void *Ax[4], *Bx[4];
   long long ldax[4], ldbx[4];
   int Kx[4];
+  // CTA-pair kernel only: the MLP's gating fused into the epilogue.
+  //   epi_mode 1, "gate | up" forward: one problem computes both projections of the same input.  A (and Aext =
+  //     s*U_gate, Aext1 = s*U_up) as usual; B, Bext describe the gate projection (W_gate [N, K], B_gate [N, Kext]),
+  //     B1, Bext1 the up projection; N = d_ff.  Outputs, all [M, N] bf16 row-major with pitch out_s0:
+  //     out = gate, out1 = up (the pre-activations, kept for the backward), out2 = h = SiLU(gate) * up.
+  //   epi_mode 2, input gradient of the down projection with the gating's backward: D = dh is not stored;
+  //     out = dgate = dh * up * SiLU'(gate), out1 = dup = dh * SiLU(gate), read from epi_in0 = gate, epi_in1 = up
+  //     ([M, N] bf16, pitch out_s0).
+  int epi_mode;
+  const void *B1, *Bext1, *Aext1;
+  long long ldb1, ldbext1, ldaext1;
+  void *out1, *out2;
+  const void *epi_in0, *epi_in1;
   // tc_decode_cluster only: role 0 = y of a projection, 1 = its u = A x^T (stored as bf16(epi_scale * u));
   // flag = the projection's index within the launch
   int role, flag;

@@ -72,6 +72,12 @@ struct alignas(64) DevProb {
   long long epi_mask_pitch;
   float epi_scale;
   int pad3;
+  // CTA-pair kernel, gating fused into the epilogue (TcProblem::epi_mode).  Mode 1 keeps the up projection's
+  // operand maps in tmXb[1] (W_up), tmXa[0] / tmXb[0] (s*U_up, B_up: the extra pair) and the maps of its further
+  // outputs in tmXa[1] (up) and tmXa[2] (h); mode 2 keeps the map of dup in tmXa[1].  Output maps of these modes
+  // have boxes of 32 rows x 32 columns, not swizzled.
+  const __nv_bfloat16 *epi_in0, *epi_in1;
+  int epi_mode, pad4;
 };
 struct DevGroup {
   DevProb p[kTcMaxProblems];
@@ -723,6 +729,7 @@ constexpr int kStage = kStageA + kStageB;        // 32 KB per CTA and stage
 // buffer (128-byte rows, 128-byte swizzle) and hands it to a bulk tensor store, so that global memory is
 // written in whole 128-byte row segments; two buffers per warp, so the next chunk is converted while the
 // previous one drains.
+constexpr int kRowsBeyond = 1 << 28;             // a row coordinate past any tensor: the copy delivers zeros
 constexpr int kOutBox = 32 * 64 * 2;             // 4 KB
 constexpr int kOutStaging = 4 * 2 * kOutBox;     // 32 KB per CTA
 constexpr int kSmemBytes = kStages * kStage + kOutStaging + 1024 + 1024;
@@ -903,7 +910,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
         const Item it = decode_item_pair(g, item);
         const DevProb &q = g.p[it.p];
         const int m0 = it.m0 + (int)rank * 128;          // this CTA's rows of the A operand
-        const int n0 = it.nt * 256 + (int)rank * 128;    // this CTA's half of the B operand
+        // this CTA's half of the B operand: 128 of the tile's 256 columns - or, for a "gate | up" problem, the
+        // tile's 128 rows of this CTA's own projection (even CTA: gate, odd CTA: up)
+        const bool gate_up = q.epi_mode == 1;
+        const int n0 = gate_up ? it.nt * 128 : it.nt * 256 + (int)rank * 128;
         const int pa_mn = q.a_mn, pb_mn = q.b_mn;
         const int nmain = it.kb1 - it.kb0;
         const int nkb = nmain + it.next;
@@ -926,7 +936,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
             }
           } else {
             if (!pb_mn) {
-              tma_load_2d_pair(sB, mb, fb, kel, n0);
+              int nrow = n0;
+              if (gate_up) {
+                // main blocks: each CTA its own frozen weight; the rank-r blocks of a projection meet zeros in
+                // the other projection's half (rows beyond the tensor are filled with zeros by the copy)
+                if (cur.seg == 0) { if (rank) mb = &q.tmXb[1]; }
+                else if ((cur.seg == 1) == (rank == 1)) nrow = kRowsBeyond;
+              }
+              tma_load_2d_pair(sB, mb, fb, kel, nrow);
             } else {
 #pragma unroll
               for (int b = 0; b < 2; ++b) tma_load_2d_pair(sB + b * 8192, mb, fb, n0 + b * 64, kel);
@@ -1010,7 +1027,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       if (item >= g.n_items) break;
       const Item it = decode_item_pair(g, item);
       const DevProb &q = g.p[it.p];
-      const int n0 = it.nt * 256;
+      const int n0 = q.epi_mode == 1 ? it.nt * 128 : it.nt * 256;
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, g.status, 600)) { ok = false; break; }
@@ -1018,6 +1035,83 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
       const int row0 = it.m0 + (int)rank * 128 + quarter * 32;   // first of this warp's 32 rows
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 256);
       uint32_t v[32], w[32];
+      if (q.epi_mode != 0) {
+        // Gating fused into the epilogue.  32 columns at a time: the accumulator values (and, backwards, the saved
+        // gate and up values of the same elements) are combined in registers, every output gets a 32 x 32 bf16 box
+        // (64-byte rows, not swizzled) in this warp's staging area, and bulk tensor stores write the boxes out.
+        const bool fwd = q.epi_mode == 1;
+        const int row = row0 + lane;
+#pragma unroll 1
+        for (int c0 = 0; c0 < (fwd ? 128 : 256); c0 += 32) {
+          const int col = n0 + c0;
+          tmem_ld32(t_row + c0, v);                              // forward: gate; backward: dh
+          if (fwd) tmem_ld32(t_row + 128 + c0, w);               // forward: up
+          uint4 gq[4], uq[4];
+          if (!fwd) {                                            // backward: saved gate and up, 64 bytes each
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              gq[j] = make_uint4(0u, 0u, 0u, 0u); uq[j] = gq[j];
+              if (row < q.M && col + 8 * j + 8 <= q.N) {
+                const long long off = (long long)row * q.out_s0 + col + 8 * j;
+                gq[j] = *reinterpret_cast<const uint4 *>(q.epi_in0 + off);
+                uq[j] = *reinterpret_cast<const uint4 *>(q.epi_in1 + off);
+              }
+            }
+          }
+          if (lane == 0) bulk_wait_group_read<0>();              // the previous boxes have been read out
+          tmem_ld_wait();
+          __syncwarp();
+          const uint32_t box0 = my_stage + (uint32_t)lane * 64u, box1 = box0 + 2048u, box2 = box0 + 4096u;
+          if (fwd) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t hh[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float gv = __uint_as_float(v[8 * j + e]), uv = __uint_as_float(w[8 * j + e]);
+                hh[e] = __float_as_uint(gv * __fdividef(1.f, 1.f + __expf(-gv)) * uv);
+              }
+              st_shared_v4(box0 + 16u * j, pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                           pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+              st_shared_v4(box1 + 16u * j, pack_bf16x2(w[8 * j], w[8 * j + 1]), pack_bf16x2(w[8 * j + 2], w[8 * j + 3]),
+                           pack_bf16x2(w[8 * j + 4], w[8 * j + 5]), pack_bf16x2(w[8 * j + 6], w[8 * j + 7]));
+              st_shared_v4(box2 + 16u * j, pack_bf16x2(hh[0], hh[1]), pack_bf16x2(hh[2], hh[3]), pack_bf16x2(hh[4], hh[5]),
+                           pack_bf16x2(hh[6], hh[7]));
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&gq[j]);
+              const __nv_bfloat162 *u2 = reinterpret_cast<const __nv_bfloat162 *>(&uq[j]);
+              uint32_t dg[8], du[8];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float2 gf = __bfloat1622float2(g2[e]), uf = __bfloat1622float2(u2[e]);
+                const float d0 = __uint_as_float(v[8 * j + 2 * e]), d1 = __uint_as_float(v[8 * j + 2 * e + 1]);
+                const float s0 = __fdividef(1.f, 1.f + __expf(-gf.x)), s1 = __fdividef(1.f, 1.f + __expf(-gf.y));
+                dg[2 * e] = __float_as_uint(d0 * uf.x * s0 * (1.f + gf.x * (1.f - s0)));
+                dg[2 * e + 1] = __float_as_uint(d1 * uf.y * s1 * (1.f + gf.y * (1.f - s1)));
+                du[2 * e] = __float_as_uint(d0 * gf.x * s0);
+                du[2 * e + 1] = __float_as_uint(d1 * gf.y * s1);
+              }
+              st_shared_v4(box0 + 16u * j, pack_bf16x2(dg[0], dg[1]), pack_bf16x2(dg[2], dg[3]), pack_bf16x2(dg[4], dg[5]),
+                           pack_bf16x2(dg[6], dg[7]));
+              st_shared_v4(box1 + 16u * j, pack_bf16x2(du[0], du[1]), pack_bf16x2(du[2], du[3]), pack_bf16x2(du[4], du[5]),
+                           pack_bf16x2(du[6], du[7]));
+            }
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && row0 < q.M && col < q.N) {
+            tma_store_2d(&q.tmOut, my_stage, col, row0);
+            tma_store_2d(&q.tmXa[1], my_stage + 2048u, col, row0);
+            if (fwd) tma_store_2d(&q.tmXa[2], my_stage + 4096u, col, row0);
+            bulk_commit_group();
+          }
+        }
+        if (lane == 0) bulk_wait_group_read<0>();   // the plain path below alternates buffers on its own count
+        __syncwarp();
+      } else
 #pragma unroll 1
       for (int c0 = 0; c0 < 256; c0 += 64, ++chunk_no) {
         tmem_ld32(t_row + c0, v);
@@ -1550,21 +1644,24 @@ EncodeTiledFn encode_fn() {
 struct MapKey {
   const void *ptr;
   long long inner, outer, pitch;
-  int box_outer;
+  int box_outer, box_inner;   // box_inner 64: 128-byte swizzle (operand tiles, plain outputs); 32: not swizzled
   bool operator==(const MapKey &o) const {
-    return ptr == o.ptr && inner == o.inner && outer == o.outer && pitch == o.pitch && box_outer == o.box_outer;
+    return ptr == o.ptr && inner == o.inner && outer == o.outer && pitch == o.pitch && box_outer == o.box_outer &&
+           box_inner == o.box_inner;
   }
 };
 struct MapKeyHash {
   size_t operator()(const MapKey &k) const {
     size_t h = reinterpret_cast<size_t>(k.ptr) * 0x9E3779B97F4A7C15ull;
-    h ^= (size_t)k.inner * 0xC2B2AE3D27D4EB4Full + (size_t)k.outer * 0x165667B19E3779F9ull + (size_t)k.pitch * 31 + (size_t)k.box_outer;
+    h ^= (size_t)k.inner * 0xC2B2AE3D27D4EB4Full + (size_t)k.outer * 0x165667B19E3779F9ull + (size_t)k.pitch * 31 +
+         (size_t)k.box_outer + 1024u * (size_t)k.box_inner;
     return h ^ (h >> 29);
   }
 };
-bool make_map(CUtensorMap *m, const void *ptr, long long inner, long long outer, long long pitch, int box_outer) {
+bool make_map(CUtensorMap *m, const void *ptr, long long inner, long long outer, long long pitch, int box_outer,
+              int box_inner = 64) {
   static thread_local std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
-  const MapKey key{ptr, inner, outer, pitch, box_outer};
+  const MapKey key{ptr, inner, outer, pitch, box_outer, box_inner};
   auto it = cache.find(key);
   if (it != cache.end()) {
     *m = it->second;
@@ -1574,11 +1671,11 @@ bool make_map(CUtensorMap *m, const void *ptr, long long inner, long long outer,
   if (!fn) return false;
   cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
   cuuint64_t gstr[1] = {(cuuint64_t)pitch * 2};
-  cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
+  cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
   cuuint32_t estr[2] = {1u, 1u};
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), gdim, gstr, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   if (cache.size() >= 8192) cache.clear();
   cache.emplace(key, *m);
@@ -1790,6 +1887,7 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
     int s = p.splits < 1 ? 1 : p.splits;
     long long w = (kb + s - 1) / s + (p.Kext + BK - 1) / BK;
     for (int e = 0; e < p.n_extra; ++e) w += (p.Kx[e] + BK - 1) / BK;
+    if (p.epi_mode == 1) w += (p.Kext + BK - 1) / BK;
     return w;
   };
   for (int i = 1; i < n && order_mode == 0; ++i)
@@ -1816,6 +1914,20 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
       return TEMPLORA_ERR_UNSUPPORTED;   // the pair kernel writes bf16 rows through bulk tensor stores
     q.m_tiles = (p.M + tile_m - 1) / tile_m;
     q.n_tiles = (p.N + BN - 1) / BN;
+    q.epi_mode = p.epi_mode; q.pad4 = 0;
+    q.epi_in0 = reinterpret_cast<const __nv_bfloat16 *>(p.epi_in0);
+    q.epi_in1 = reinterpret_cast<const __nv_bfloat16 *>(p.epi_in1);
+    if (p.epi_mode != 0) {
+      if (!use_pair || p.epi_mode < 0 || p.epi_mode > 2 || p.n_extra != 0 || !p.out1) return TEMPLORA_ERR_UNSUPPORTED;
+      if (p.epi_mode == 1) {
+        if (p.a_mn || p.b_mn || p.Kext <= 0 || !p.B1 || !p.Bext1 || !p.Aext1 || !p.out2 ||
+            ((p.ldb1 | p.ldbext1 | p.ldaext1) & 7))
+          return TEMPLORA_ERR_INVALID_ARG;
+        q.n_tiles = (p.N + 127) / 128;   // a tile holds 128 columns of gate and the same 128 columns of up
+      } else if (!p.epi_in0 || !p.epi_in1 || ((reinterpret_cast<uintptr_t>(p.epi_in0) | reinterpret_cast<uintptr_t>(p.epi_in1)) & 15)) {
+        return TEMPLORA_ERR_INVALID_ARG;
+      }
+    }
     q.item_start = items;
     q.a_mn = p.a_mn; q.b_mn = p.b_mn;
     q.out_f32 = p.out_f32; q.pad = 0;
@@ -1848,8 +1960,22 @@ templora_status_t tc_gemm_grouped(const TcProblem *probs, int n, int BN, DeviceS
       ok = ok && make_operand_map(&q.tmXa[e], p.Ax[e], p.M, p.Kx[e], p.ldax[e], p.a_mn, BM) &&
            make_operand_map(&q.tmXb[e], p.Bx[e], p.N, p.Kx[e], p.ldbx[e], p.b_mn, box_b);
     }
-    if (use_pair) ok = ok && make_map(&q.tmOut, p.out, p.N, p.M, p.out_s0, 32);
+    if (use_pair && p.epi_mode == 0) ok = ok && make_map(&q.tmOut, p.out, p.N, p.M, p.out_s0, 32);
     else q.tmOut = q.tmA;
+    if (p.epi_mode != 0) {
+      if ((reinterpret_cast<uintptr_t>(p.out1) & 15) || (p.out2 && (reinterpret_cast<uintptr_t>(p.out2) & 15)))
+        return TEMPLORA_ERR_INVALID_ARG;
+      ok = ok && make_map(&q.tmOut, p.out, p.N, p.M, p.out_s0, 32, 32) &&
+           make_map(&q.tmXa[1], p.out1, p.N, p.M, p.out_s0, 32, 32);
+      if (p.epi_mode == 1) {
+        q.kb_x[0] = q.kb_ext;
+        q.kb_xtot = q.kb_ext;
+        ok = ok && make_map(&q.tmXa[2], p.out2, p.N, p.M, p.out_s0, 32, 32) &&
+             make_operand_map(&q.tmXb[1], p.B1, p.N, p.K, p.ldb1, 0, box_b) &&
+             make_operand_map(&q.tmXa[0], p.Aext1, p.M, p.Kext, p.ldaext1, 0, BM) &&
+             make_operand_map(&q.tmXb[0], p.Bext1, p.N, p.Kext, p.ldbext1, 0, box_b);
+      }
+    }
     if (!ok) return TEMPLORA_ERR_CUDA;
   }
   g.n_items = items;
@@ -1895,6 +2021,7 @@ templora_status_t tc_decode_cluster(const TcProblem *probs, int n, int n_tokens,
     q.kb_xtot = 0;
     for (int e = 0; e < kMaxExtra; ++e) { q.kb_x[e] = 0; q.tmXa[e] = q.tmA; q.tmXb[e] = q.tmB; }
     q.tmOut = q.tmA;
+    q.epi_mode = 0; q.pad4 = 0; q.epi_in0 = nullptr; q.epi_in1 = nullptr;
     q.epi_mask = nullptr; q.epi_mask_pitch = 0; q.epi_scale = p.epi_scale;
     q.out = p.out; q.out_s0 = 1; q.out_s1 = p.out_s1; q.out_split = 0;
     items += q.m_tiles;

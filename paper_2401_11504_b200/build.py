@@ -36,6 +36,7 @@ def build_library(force=False, verbose=False):
         return LIB
     cmd = [_nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "--threads", "4", "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    cmd += os.environ.get("TEMPLORA_NVCC_FLAGS", "").split()   # e.g. -DTL_SK_CHUNK_MB=16 to try a tuning macro
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]

@@ -19,6 +19,8 @@
 // a launch is balanced whatever the mix of long and short items.  The counter must be zero at
 // launch (the workspace head is zeroed once by the caller); the last CTA to finish resets it.
 #include "common.cuh"
+#include "tc_device.cuh"
+#include "tc_host.h"
 
 #include <cuda.h>
 
@@ -29,11 +31,9 @@
 namespace templora {
 namespace {
 
-constexpr int BM = 128, BK = 64;
 constexpr int kThreads = 192;
 constexpr int kThreads2 = 224;   // single-CTA GEMM kernel: one more warp, the second TMA producer
 constexpr int kSched = 4;  // depth of the work-item ring between the producer and its consumers
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 constexpr int kStageA = BM * BK * 2;  // 16 KB
 // KPS = k-blocks per pipeline stage.  The decode stream (BN = 16) moves two k-blocks per stage so that
@@ -89,162 +89,6 @@ struct Item {
   int p, m0, nt, split, kb0, kb1, next;
 };
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when the CTA is aborting or the limit ran out (then it also
-// raises the CTA's abort flag and records the location in the device status record).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, DeviceStatus *st,
-                                       int where) {
-  for (int i = 0; i < 4096; ++i)
-    if (mbar_try(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
-  while (true) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1;
-      if (st && atomicCAS(&st->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) st->where = where;
-      __threadfence();
-      return false;
-    }
-  }
-}
-
-// Fast path of a wait: one poll inline, the bounded loop only when the barrier is not ready yet.
-__device__ __forceinline__ bool mbar_wait_fast(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                               DeviceStatus *st, int where) {
-  if (mbar_try(bar, parity)) return true;
-  return mbar_wait(bar, parity, abort_flag, st, where);
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-      : "memory");
-}
-
-// Same load with an L2 eviction-priority hint (a 64-bit policy from createpolicy).
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
-                                                 uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
-      : "memory");
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-
-// Bulk tensor store of one box from shared memory (written by this warp through the generic proxy, made
-// visible with fence_proxy_async_smem) to global memory; elements outside the tensor are not written.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// at most N of this thread's bulk groups may still be reading their shared-memory source
-template <int N> __device__ __forceinline__ void bulk_wait_group_read() {
-  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo_f32, uint32_t hi_f32) {
-  __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(lo_f32), __uint_as_float(hi_f32));
-  return *reinterpret_cast<uint32_t *>(&t);
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// Shared-memory matrix descriptor, 128-byte swizzle.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= 1ull << 46;  // descriptor version for tcgen05
-  d |= 2ull << 61;  // 128-byte swizzle
-  return d;
-}
-// Descriptor of an operand tile with the start-address field left zero, and the start-address step
-// (in 16-byte units) from one K = 16 slice to the next.  K-contiguous tiles advance 32 bytes inside
-// the 128-byte swizzled row; M/N-contiguous tiles advance two 8-row groups (2048 bytes).
-__device__ __forceinline__ uint64_t smem_desc_template(int mn_major) {
-  return mn_major ? smem_desc(0, 8192, 1024) : smem_desc(0, 16, 1024);
-}
-__device__ __forceinline__ uint32_t smem_desc_kstep(int mn_major) { return mn_major ? (2048u >> 4) : (32u >> 4); }
-
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc(int n, int a_mn, int b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
-      "%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ Item decode_item(const DevGroup &g, int item) {
   int p = 0;
@@ -1621,6 +1465,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 }  // namespace dcl
 
 
+}  // namespace
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -1659,7 +1505,7 @@ struct MapKeyHash {
   }
 };
 bool make_map(CUtensorMap *m, const void *ptr, long long inner, long long outer, long long pitch, int box_outer,
-              int box_inner = 64) {
+              int box_inner) {
   static thread_local std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
   const MapKey key{ptr, inner, outer, pitch, box_outer, box_inner};
   auto it = cache.find(key);
@@ -1700,13 +1546,6 @@ int stream_sm_limit(cudaStream_t st, int sm_count) {
   return it->second;
 }
 
-struct DeviceInfo {
-  int sm_count = 0;
-  int cc_major = 0;
-  bool attr_set[3] = {false, false, false};
-  bool pair_attr_set = false;
-  int dcl_clusters[4] = {};   // per decode-cluster kernel variant: clusters that fit at once (0 = not asked yet, -1 = none)
-};
 DeviceInfo *device_info() {
   static DeviceInfo info[64];
   int dev = 0;
@@ -1721,6 +1560,8 @@ DeviceInfo *device_info() {
   }
   return &d;
 }
+
+namespace {
 
 template <int BN>
 templora_status_t launch(const DevGroup &g, DeviceInfo *di, int slot, cudaStream_t st) {

@@ -538,8 +538,19 @@ def config_70b(b, torch, inputs, runtime, dev, peaks, hp, steps=12, warmup=3):
 def parallel_deployment(b, torch, runtime, blk, hp, update_sms=116, decode_sms=32, n_updates=20):
     """The paper's parallelized deployment on one GPU: chunk updates (7B block, T=1024) back to back on
     one stream while single-token decode steps of the same block run on another, with the SMs split
-    between the two persistent kernels.  Reports both rates alone and side by side."""
-    dep = runtime.ParallelDeployment(b, blk, n_tokens=1, update_sms=update_sms, decode_sms=decode_sms)
+    between the two sides: fixed disjoint groups of SMs (templora_sm_partition_create) and, for comparison,
+    per-stream caps on the grid sizes alone.  Reports both rates alone and side by side."""
+    out = _parallel_deployment(b, torch, runtime, blk, hp, update_sms, decode_sms, n_updates, True)
+    if out["sm_partition"]:
+        caps = _parallel_deployment(b, torch, runtime, blk, hp, update_sms, decode_sms, n_updates, False)
+        out["caps_only"] = {k: caps[k] for k in ("update_ms_alone_capped", "decode_step_us_alone_capped",
+                                                 "update_ms_side_by_side", "decode_step_us_side_by_side")}
+    return out
+
+
+def _parallel_deployment(b, torch, runtime, blk, hp, update_sms, decode_sms, n_updates, partition):
+    dep = runtime.ParallelDeployment(b, blk, n_tokens=1, update_sms=update_sms, decode_sms=decode_sms,
+                                     partition=partition)
     ev = lambda: torch.cuda.Event(enable_timing=True)
     try:
         def timed(fn, stream, reps):
@@ -575,12 +586,13 @@ def parallel_deployment(b, torch, runtime, blk, hp, update_sms=116, decode_sms=3
         dec_side_us = (ends[contended[-1]] / (contended[-1] + 1) * 1e3) if contended else None
         dep.publish()
         torch.cuda.synchronize()
-        return {"update_sms": update_sms, "decode_sms": decode_sms,
+        return {"update_sms": dep.update_sms, "decode_sms": dep.decode_sms, "sm_partition": dep.partition is not None,
                 "update_ms_alone_capped": upd_alone_ms, "decode_step_us_alone_capped": dec_alone_ms * 1e3,
                 "update_ms_side_by_side": e0.elapsed_time(e1) / n_updates,
                 "decode_step_us_side_by_side": dec_side_us, "decode_steps_during_updates": len(contended),
                 "what": "7B block: chunk updates (T=1024) back to back on one stream, single-token decode steps of the "
-                        "same block on another; 'alone' figures keep the SM caps"}
+                        "same block on another; 'alone' figures keep the SM split; caps_only: ordinary streams with "
+                        "per-stream caps on the persistent kernels' grids instead of disjoint SM groups"}
     finally:
         dep.close()
 

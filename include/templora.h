@@ -2,8 +2,8 @@
  * templora.h -- C ABI of the B200 (sm_100a) Temp-Lora chunk-update library.
  *
  * The library runs the per-chunk inference-time update of a temporary LoRA
- * module ("Train Theta_k: In X_T -> Out Chunk_k (n epochs, learning rate alpha)",
- * Algorithm 1 of the Temp-Lora paper) for LoRA-augmented linear projections, and
+ * module (Algorithm 1 of the Temp-Lora paper, the training step of the module Theta_k;
+ * hyper-parameters of the "Setup" paragraph) for LoRA-augmented linear projections, and
  * the decode-time forward used between updates (Algorithm 1, generation step).
  *
  * Notation (row-major, contiguous rows, no bias):
@@ -27,8 +27,9 @@
  *     generic kernel path.  r <= 256 always (the paper sweeps rank 16..256).
  *   - Workspace: 256-byte aligned, at least templora_*workspace_bytes() long, and its
  *     first 1024 bytes zeroed by the caller once before first use (they hold the
- *     device status record).  A workspace must not be shared by calls that may
- *     overlap on the GPU.
+ *     device status record and the kernels' work counters and flags, which every
+ *     kernel leaves at zero; zero them again after a TEMPLORA_ERR_TIMEOUT was
+ *     recorded).  A workspace must not be shared by calls that may overlap on the GPU.
  *   - Synchronous errors (bad argument, unsupported shape, short workspace, a CUDA
  *     launch failure) are returned and nothing further is launched.  Device-side
  *     problems (a bounded wait inside a kernel ran out) are recorded in the status
@@ -103,7 +104,7 @@ size_t templora_update_block_workspace_bytes(const templora_linear_t *proj, int3
 
 /*
  * Forward of the LoRA-augmented projection over a chunk of T tokens
- * (module forward inside "Train Theta_k", Algorithm 1; LoRA of the Section "Temp-Lora"):
+ * (module forward inside the training step of Theta_k, Algorithm 1; LoRA of the Section "Temp-Lora"):
  *     U = x A^T ;  y = x W0^T + s U B^T
  * (with dropout_p > 0:  U = xd A^T,  xd = x * keep / (1 - p))
  * x [T,d_in] in, y [T,d_out] out.  U_save: optional fp32 [T,r] that receives U
@@ -127,7 +128,7 @@ templora_status_t templora_linear_bwd(const templora_linear_t *lin, int32_t T, c
 
 /*
  * One AdamW step (decoupled weight decay, bias-corrected) on n_params tensors
- * (optimizer step of "Train Theta_k"; learning rate 5e-5 in the paper's Setup,
+ * (optimizer step of the training step of Theta_k, Algorithm 1; learning rate 5e-5 in the paper's Setup,
  * fp32 master weights and moments as bfloat16 ZeRO-2 training implies):
  *     p <- p (1 - lr wd);  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2
  *     p <- p - lr (m / (1-b1^step)) / (sqrt(v / (1-b2^step)) + eps)
@@ -225,7 +226,7 @@ const char *templora_status_string(templora_status_t st);
 templora_status_t templora_read_device_status(void *ws, void *stream, int32_t *code, int32_t *where);
 
 /*
- * The element-wise steps on either side of the projections when "Train Theta_k" (Algorithm 1) runs over
+ * The element-wise steps on either side of the projections when the training step of Theta_k (Algorithm 1) runs over
  * a Llama-style decoder block: the MLP's gating between gate/up and down, and the RMSNorm in front of
  * q,k,v and of gate,up.  The paper names neither (it trains stock Llama-2 / Yi blocks); the formulas are
  * those models' definitions.  All tensors are contiguous DEVICE buffers of `dtype` (templora_dtype_t),
@@ -251,7 +252,7 @@ templora_status_t templora_rmsnorm_bwd(int32_t T, int32_t d, int32_t dtype, cons
                                        float eps, void *dx, void *stream);
 
 /*
- * The chunk update of the MLP of a Llama-style decoder block in one call ("Train Theta_k", Algorithm 1, run over
+ * The chunk update of the MLP of a Llama-style decoder block in one call (the training step of Theta_k, Algorithm 1, run over
  * the block's gate, up and down projections with the gating between them; the gating is the model's, see above):
  *     gate = x Wg^T + s (x Ag^T) Bg^T     up = x Wu^T + s (x Au^T) Bu^T     h = SiLU(gate) * up
  *     y    = h Wd^T + s (h Ad^T) Bd^T
@@ -291,6 +292,28 @@ templora_status_t templora_selftest_bounded_wait(void *ws, size_t ws_bytes, int3
  * max_sms = 0 removes the cap.  Process-wide table keyed by the stream handle.
  */
 templora_status_t templora_set_stream_sm_limit(void *stream, int32_t max_sms);
+
+/*
+ * Parallelized deployment with disjoint SMs ("Further Analysis", same passage).  A cap alone bounds how many SMs a
+ * stream's kernels ask for, not which ones, so the two sides still get in each other's way at every kernel
+ * boundary.  templora_sm_partition_create splits the current device's SMs into two fixed groups and creates one
+ * stream in each (driver green contexts): kernels launched on stream_first only ever run on the first group's
+ * SMs, those on stream_rest on the others.  first_sms is rounded by the driver to its granularity (8 SMs on
+ * sm_100); sms_first / sms_rest report what each side got, and the matching per-stream caps are set.
+ *   - `out` is a HOST struct filled by the call; the streams are cudaStream_t handles owned by the partition
+ *     (non-blocking with respect to the legacy default stream) and may be used with any CUDA call.
+ *   - Device memory, tensor maps and workspaces are shared with the rest of the process as usual.
+ *   - TEMPLORA_ERR_UNSUPPORTED when the driver offers no SM partitioning; nothing is created then.
+ *   - templora_sm_partition_destroy synchronises both streams, destroys them and releases the groups.
+ */
+typedef struct {
+  void *handle;          /* opaque */
+  void *stream_first;    /* cudaStream_t */
+  void *stream_rest;     /* cudaStream_t */
+  int32_t sms_first, sms_rest;
+} templora_sm_partition_t;
+templora_status_t templora_sm_partition_create(int32_t first_sms, templora_sm_partition_t *out);
+templora_status_t templora_sm_partition_destroy(templora_sm_partition_t *part);
 
 /*
  * Kernel-path selection for testing: 0 = automatic (tensor-core path when the

@@ -5,8 +5,8 @@ CUDA library is checked against.  It shares no code with the CUDA path and is
 imported only by the tests, by the smoke check and by the CPU-baseline leg of
 the benchmark.  The product never calls it.
 
-What it computes (Temp-Lora, Section "Temp-Lora" and Algorithm 1, step
-"Train Theta_k ... (n epochs, learning rate alpha)"; the module is the LoRA
+What it computes (Temp-Lora, Section "Temp-Lora" and Algorithm 1, the training
+step of the module Theta_k over a chunk; the module is the LoRA
 module of Hu et al. that the paper adopts by citation, with the hyper-parameters
 of the paper's "Setup" paragraph: alpha = 64, rank = 64, learning rate 5e-5,
 n = 2 epochs, bfloat16 training):
@@ -259,7 +259,7 @@ def update_block(projs, epochs, lr, beta1, beta2, eps, weight_decay, step0=0, bf
 
 # ---------------------------------------------------------------------------
 # The steps on either side of the projections inside a decoder block's update
-# ("Train Theta_k" runs a whole Llama-style block: RMSNorm -> q,k,v ... and
+# (the training step of Theta_k, Algorithm 1, runs a whole Llama-style block: RMSNorm -> q,k,v ... and
 # gate, up -> SiLU(gate) * up -> down).  Plain definitions, fp64.
 # ---------------------------------------------------------------------------
 def swiglu_fwd(gate, up):

@@ -25,12 +25,18 @@ EXPORTS = [
     "templora_set_stream_sm_limit", "templora_selftest_bounded_wait", "templora_lr_at_step",
     "templora_update_block_warmup", "templora_swiglu_fwd", "templora_swiglu_bwd", "templora_rmsnorm_fwd",
     "templora_rmsnorm_bwd", "templora_decode_fwd_noalloc_status", "templora_update_mlp",
-    "templora_update_mlp_workspace_bytes",
+    "templora_update_mlp_workspace_bytes", "templora_sm_partition_create", "templora_sm_partition_destroy",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 (KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
  KIND_TC_DROPOUT_TERM, KIND_BLOCK_OPS) = range(10)
 N_KINDS = 10
+
+
+class SmPartition(C.Structure):
+    """templora_sm_partition_t: two streams whose kernels run on disjoint groups of SMs."""
+    _fields_ = [("handle", C.c_void_p), ("stream_first", C.c_void_p), ("stream_rest", C.c_void_p),
+                ("sms_first", C.c_int32), ("sms_rest", C.c_int32)]
 
 
 class LinearDesc(C.Structure):
@@ -98,6 +104,10 @@ def _load():
     lib.templora_selftest_bounded_wait.argtypes = [vp, sz, i32, vp]
     lib.templora_set_stream_sm_limit.restype = i32
     lib.templora_set_stream_sm_limit.argtypes = [vp, i32]
+    lib.templora_sm_partition_create.restype = i32
+    lib.templora_sm_partition_create.argtypes = [i32, C.POINTER(SmPartition)]
+    lib.templora_sm_partition_destroy.restype = i32
+    lib.templora_sm_partition_destroy.argtypes = [C.POINTER(SmPartition)]
     lib.templora_status_string.restype = C.c_char_p
     lib.templora_status_string.argtypes = [i32]
     lib.templora_read_device_status.restype = i32
@@ -373,6 +383,18 @@ def templora_decode_block_fwd(args, ws, stream=None):
 def templora_set_stream_sm_limit(stream, max_sms):
     """Cap the SMs the persistent kernels use on `stream` (0 = no cap)."""
     _check(lib.templora_set_stream_sm_limit(_stream(stream), int(max_sms)), "templora_set_stream_sm_limit")
+
+
+def templora_sm_partition_create(first_sms):
+    """Split the current device's SMs into two groups with one stream each; returns the filled SmPartition
+    (wrap its streams with torch.cuda.ExternalStream to use them from torch)."""
+    part = SmPartition()
+    _check(lib.templora_sm_partition_create(int(first_sms), C.byref(part)), "templora_sm_partition_create")
+    return part
+
+
+def templora_sm_partition_destroy(part):
+    _check(lib.templora_sm_partition_destroy(C.byref(part)), "templora_sm_partition_destroy")
 
 
 def templora_selftest_bounded_wait(ws, limit_ms=50, stream=None):

@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtemplora.so")
-SOURCES = ["api.cu", "tc_gemm.cu", "simt_gemm.cu", "elementwise.cu", "block_ops.cu", "timing.cu", "decode_noalloc.cu"]
+SOURCES = ["api.cu", "tc_gemm.cu", "simt_gemm.cu", "elementwise.cu", "block_ops.cu", "timing.cu", "decode_noalloc.cu", "sm_partition.cu"]
 
 
 def _nvcc():

@@ -1022,7 +1022,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 // (deterministic) and writes y.  The rank-r term rides in the same accumulators as extension k-blocks
 // (B tile x (s u)^T) at the end of the tile's k-block sequence.  u = A x^T is itself one more item per
 // projection (the rows of A as the streamed operand): its cluster writes s*u as bf16 to scratch and
-// raises a flag (the launch's epoch number) that the other clusters' producers check before they
+// raises a flag (zero again when the launch ends) that the other clusters' producers check before they
 // load extension operands.  The u items are dealt first, so each is the first item of its cluster
 // and waits for nothing.  Items are handed out dynamically: CTA 0's producer draws them from a global
 // counter and writes them into every CTA's item ring.
@@ -1052,7 +1052,7 @@ constexpr int kRing = 8;    // items the dealer may run ahead of the slowest rea
 // extension A-op B, B-op s*u; out = y [n, d_out] bf16), 1 = its u (A-op A, B-op x; out = s*u [n, r] bf16,
 // scale in epi_scale); DevProb::pad3 = the projection's slot among the ready flags.
 struct DclParams {
-  int n_tokens, epoch, n_stages;
+  int n_tokens, n_stages;
 };
 
 __device__ __forceinline__ int4 ld_volatile_i4(const int *p) {
@@ -1254,7 +1254,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             while (true) {
               const int f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
 #pragma unroll
-              for (int w = 0; w < 8; ++w) ready_mask |= (f[w] == prm.epoch ? 1u : 0u) << w;
+              for (int w = 0; w < 8; ++w) ready_mask |= (f[w] != 0 ? 1u : 0u) << w;
               if ((ready_mask >> q.pad3) & 1u) break;
               f0 = ld_volatile_i4(flags); f1 = ld_volatile_i4(flags + 4);
               if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
@@ -1436,7 +1436,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (atomicAdd(arrived, 1) == 3) {
             *arrived = 0;
             __threadfence();
-            st_release_gpu(flags + q.pad3, prm.epoch);
+            st_release_gpu(flags + q.pad3, 1);
           }
         }
       }
@@ -1450,11 +1450,13 @@ __global__ void __launch_bounds__(kThreads, 1)
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
   }
-  // the last cluster to finish re-arms the item counter for the next launch on this workspace
+  // the last cluster to finish re-arms the item counter and the ready flags for the next launch on this
+  // workspace (nothing of the launch depends on a number the host hands in, so a recorded launch can be replayed)
   if (rank == 0 && threadIdx.x == 0) {
     __threadfence();
     const int done = atomicAdd(&g.status->sched_done, 1);
     if (done == n_clusters - 1) {
+      for (int w = 0; w < kDclMaxProj; ++w) flags[w] = 0;
       g.status->sched_next = 0;
       g.status->sched_done = 0;
       __threadfence();
@@ -1878,10 +1880,8 @@ templora_status_t tc_decode_cluster(const TcProblem *probs, int n, int n_tokens,
     if (!ok) return TEMPLORA_ERR_CUDA;
   }
   g.n_items = items;
-  static std::atomic<int> epoch_counter{0};
   dcl::DclParams prm;
   prm.n_tokens = n_tokens;
-  do { prm.epoch = epoch_counter.fetch_add(1) + 1; } while (prm.epoch == 0);
   // every u item must be the first item of its cluster (it then waits for nothing): the launchers
   // below start cluster c on item c, so they need at least n_u clusters
   // 72 KB stages (four k-blocks) when three of them fit beside the receive buffer, else 36 KB stages

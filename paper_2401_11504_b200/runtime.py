@@ -246,16 +246,31 @@ class ParallelDeployment:
     on another stream and reads separate *serving* copies, so it always sees a complete module.
     publish() swaps the new module in at a decode-step boundary: on the decode stream, after the
     update's completion event, the working copies are copied over the serving copies (10 MB for a
-    7B-shaped block).  Per-stream SM caps keep both persistent kernels resident at once.
+    7B-shaped block).  The two streams run on disjoint groups of SMs (templora_sm_partition_create:
+    decode_sms for the decode stream, the rest for the update); with partition=False, or where the
+    driver offers no SM partitioning, they are ordinary streams with per-stream SM caps.
     Orchestration only: every product runs in the library's kernels.
     """
 
-    def __init__(self, b, blk, n_tokens=1, update_sms=116, decode_sms=32, device="cuda"):
+    def __init__(self, b, blk, n_tokens=1, update_sms=116, decode_sms=32, device="cuda", partition=True):
         self.b, self.blk, self.n = b, blk, n_tokens
-        self.update_stream = torch.cuda.Stream(device=device)
-        self.decode_stream = torch.cuda.Stream(device=device)
-        b.templora_set_stream_sm_limit(self.update_stream, update_sms)
-        b.templora_set_stream_sm_limit(self.decode_stream, decode_sms)
+        self.partition = None
+        if partition:
+            try:
+                self.partition = b.templora_sm_partition_create(decode_sms)
+            except b.TemploraError as e:
+                if e.code != b.ERR_UNSUPPORTED:
+                    raise
+        if self.partition is not None:
+            self.decode_stream = torch.cuda.ExternalStream(self.partition.stream_first, device=device)
+            self.update_stream = torch.cuda.ExternalStream(self.partition.stream_rest, device=device)
+            self.decode_sms, self.update_sms = self.partition.sms_first, self.partition.sms_rest
+        else:
+            self.update_stream = torch.cuda.Stream(device=device)
+            self.decode_stream = torch.cuda.Stream(device=device)
+            b.templora_set_stream_sm_limit(self.update_stream, update_sms)
+            b.templora_set_stream_sm_limit(self.decode_stream, decode_sms)
+            self.decode_sms, self.update_sms = decode_sms, update_sms
         self.serving = [(st["A"]["work"].clone(), st["B"]["work"].clone()) for st in blk.state]
         self.lins = [b.linear_desc(W0, a, bb, blk.s) for W0, (a, bb) in zip(blk.W0, self.serving)]
         td = blk.x[0].dtype
@@ -293,5 +308,9 @@ class ParallelDeployment:
         self.published.record(self.decode_stream)
 
     def close(self):
+        if self.partition is not None:
+            self.b.templora_sm_partition_destroy(self.partition)   # synchronises and destroys both streams
+            self.partition = None
+            return
         self.b.templora_set_stream_sm_limit(self.update_stream, 0)
         self.b.templora_set_stream_sm_limit(self.decode_stream, 0)

@@ -20,13 +20,16 @@ def b():
     return binding
 
 
-def test_decode_sees_old_module_until_publish(b):
+@pytest.mark.parametrize("partition", [True, False])
+def test_decode_sees_old_module_until_publish(b, partition):
+    # partition=True: the two streams own disjoint groups of SMs; False: ordinary streams with per-stream caps
     from paper_2401_11504_b200 import runtime
     shapes = [("q", 512, 512), ("gate", 512, 1408), ("down", 1408, 512)]
     hp = hp32(dict(lr=2e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0))
     blk = runtime.Block(b, 3, "pardep", shapes, 512, 64, 2.0, "bf16", "cuda")
     snap = snapshot_block(blk)
-    dep = runtime.ParallelDeployment(b, blk, n_tokens=4, update_sms=116, decode_sms=32)
+    dep = runtime.ParallelDeployment(b, blk, n_tokens=4, update_sms=116, decode_sms=32, partition=partition)
+    assert (dep.partition is not None) == partition
     try:
         xs = [f64(x) for x in dep.x]
         old = [orc.decode_fwd(x, p["W0"], p["A_master"], p["B_master"], 2.0) for x, p in zip(xs, snap)]
@@ -75,3 +78,27 @@ def test_stream_sm_limit_keeps_results(b):
             check_fwd_bwd(b, 31, "capped", 300, 512, 640, 64, 2.0, "bf16")
     finally:
         b.templora_set_stream_sm_limit(st, 0)
+
+
+def test_sm_partition_splits_the_device_and_both_streams_compute(b):
+    # the two groups cover the device's SMs between them, each stream carries the matching cap, and a
+    # forward/backward on either stream (tensors made on the default stream) matches the oracle
+    from parity_utils import check_fwd_bwd
+    total = torch.cuda.get_device_properties(0).multi_processor_count
+    part = b.templora_sm_partition_create(32)
+    try:
+        assert part.sms_first >= 32 and part.sms_rest >= 1 and part.sms_first + part.sms_rest <= total
+        assert part.sms_first % 8 == 0
+        for handle, tag in ((part.stream_first, "part-first"), (part.stream_rest, "part-rest")):
+            st = torch.cuda.ExternalStream(handle)
+            torch.cuda.synchronize()
+            with torch.cuda.stream(st):
+                check_fwd_bwd(b, 33, tag, 300, 512, 640, 64, 2.0, "bf16")
+            st.synchronize()
+    finally:
+        b.templora_sm_partition_destroy(part)
+    assert part.handle is None
+    with pytest.raises(b.TemploraError):
+        b.templora_sm_partition_create(0)
+    with pytest.raises(b.TemploraError):
+        b.templora_sm_partition_create(total)

@@ -523,40 +523,6 @@ __global__ void __launch_bounds__(kThreads2, 1) tc_gemm_kernel(const __grid_cons
   }
 }
 
-// ------------------------------------------------------------------ helpers shared by the cluster kernels
-__device__ __forceinline__ void st_cluster_s32(uint32_t addr, int v) {
-  asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-// Arrive on a peer's barrier to say "I have finished reading" (nothing of mine needs to become visible).
-__device__ __forceinline__ void mbar_arrive_remote_plain(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_acq_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait whose success also makes a peer's earlier shared-memory stores (released at cluster scope) visible.
-__device__ __noinline__ bool mbar_wait_acq_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                   DeviceStatus *st, int where) {
-  for (int i = 0; i < 4096; ++i)
-    if (mbar_try_acq_cluster(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
-  while (true) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_acq_cluster(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1;
-      if (st && atomicCAS(&st->code, 0, (int)TEMPLORA_ERR_TIMEOUT) == 0) st->where = where;
-      __threadfence();
-      return false;
-    }
-  }
-}
-
 // ------------------------------------------------------------------ CTA-pair kernel (256 x 256 tiles)
 // Two CTAs of a cluster (one TPC) share one 256 x 256 output tile: each loads its own 128 rows of
 // the A operand and its own 128-column half of the B operand, and the even CTA issues
@@ -580,23 +546,6 @@ constexpr int kSmemBytes = kStages * kStage + kOutStaging + 1024 + 1024;
 constexpr int kTmemCols = 512;                   // two 256-column accumulators
 constexpr int kPairThreads = 224;                // producer (A), MMA, four epilogue warps, producer (B)
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 // TMA load whose completion is signalled on a barrier that may live in the peer CTA of the pair.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster, int c0,
                                                  int c1) {
@@ -1055,22 +1004,6 @@ struct DclParams {
   int n_tokens, n_stages;
 };
 
-__device__ __forceinline__ int4 ld_volatile_i4(const int *p) {
-  int4 v;
-  asm volatile("ld.volatile.global.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_release_gpu(int *p, int v) {
-  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-// Remote store of 16 bytes into a peer's shared memory; the peer's mbarrier counts the bytes as they land.
-__device__ __forceinline__ void st_async_v4(uint32_t remote_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
-                                            uint32_t remote_bar) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
-               ::"r"(remote_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
-
 template <int S, int KPS>
 __global__ void __launch_bounds__(kThreads, 1)
     decode_cluster_kernel(const __grid_constant__ DevGroup g, const DclParams prm) {
@@ -1101,7 +1034,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t ring0 = bar0 + 512 + 16;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rank = (int)pair::cluster_ctarank();
+  const int rank = (int)cluster_ctarank();
   const int cluster_id = blockIdx.x / S, n_clusters = gridDim.x / S;
   int *flags = &g.status->pad[0];
   // every role but CTA 0's producer takes its items from the ring: 6 per CTA
@@ -1125,7 +1058,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
   tc_fence_before();
   __syncthreads();
-  pair::cluster_sync_all();   // the peers' barriers are initialised before anything is sent to them
+  cluster_sync_all();   // the peers' barriers are initialised before anything is sent to them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // Ordering against the kernels ahead on the stream.  Everything this kernel reads may have been written by them
@@ -1157,7 +1090,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     return true;
   };
   auto ring_release = [&](int &sslot, uint32_t &sphase) {
-    mbar_arrive_remote_plain(pair::mapa_shared(sempty_bar(sslot), 0));
+    mbar_arrive_remote_plain(mapa_shared(sempty_bar(sslot), 0));
     if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
   };
 
@@ -1175,10 +1108,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       auto deal = [&](int it) -> bool {
         if (!mbar_wait(sempty_bar(sslot), sphase ^ 1u, abort_flag, g.status, 830)) return false;
 #pragma unroll
-        for (int r = 0; r < S; ++r) st_cluster_s32(pair::mapa_shared(ring0 + 4u * sslot, (uint32_t)r), it);
+        for (int r = 0; r < S; ++r) st_cluster_s32(mapa_shared(ring0 + 4u * sslot, (uint32_t)r), it);
 #pragma unroll
         for (int r = 0; r < S; ++r)   // release at cluster scope: the store above is visible to whoever sees this arrival
-          pair::mbar_arrive_cluster(pair::mapa_shared(sfull_bar(sslot), (uint32_t)r));
+          mbar_arrive_cluster(mapa_shared(sfull_bar(sslot), (uint32_t)r));
         if (++sslot == kRing) { sslot = 0; sphase ^= 1u; }
         return true;
       };
@@ -1386,8 +1319,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         // send this row's partial sums into CTA 0's shared memory, once CTA 0 has read the previous ones
         ok = __all_sync(0xffffffffu, mbar_wait(part_free, (uint32_t)(seq & 1) ^ 1u, abort_flag, g.status, 821));
         if (!ok) break;
-        const uint32_t dst = pair::mapa_shared(recv0 + (uint32_t)((rank - 1) * slot_bytes + row_in_tile * 16 * nv), 0);
-        const uint32_t bar = pair::mapa_shared(part_full, 0);
+        const uint32_t dst = mapa_shared(recv0 + (uint32_t)((rank - 1) * slot_bytes + row_in_tile * 16 * nv), 0);
+        const uint32_t bar = mapa_shared(part_full, 0);
 #pragma unroll
         for (int c = 0; c < 4; ++c)
           if (c < nv) st_async_v4(dst + 16u * c, v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3], bar);
@@ -1415,7 +1348,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       __syncwarp();
       if (lane == 0) {
 #pragma unroll
-        for (int r = 1; r < S; ++r) mbar_arrive_remote_plain(pair::mapa_shared(part_free, (uint32_t)r));
+        for (int r = 1; r < S; ++r) mbar_arrive_remote_plain(mapa_shared(part_free, (uint32_t)r));
       }
       __syncwarp();
       const int row = m0 + row_in_tile;
@@ -1445,7 +1378,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   tc_fence_before();
   __syncthreads();
-  pair::cluster_sync_all();   // no CTA leaves while a peer may still read its partial or signal its barriers
+  cluster_sync_all();   // no CTA leaves while a peer may still read its partial or signal its barriers
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");

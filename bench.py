@@ -36,7 +36,7 @@ NOMINAL_TFLOPS = 2250.0         # dense bf16, data sheet
 # DRAM traffic of one launch of the dominant kernel (bytes), from an ncu capture summarised under
 # profiles/; valid only while the kernel source is the one that was profiled.
 SHARED_INPUTS = [["q", "k", "v"], ["gate", "up"]]   # projections of a decoder block that read the same tensor
-TRAFFIC = {"tc_gemm_sha1": "40d51c0f35237ab99937b748fc9bc0ed34ae6cba", "bytes_per_launch": 1136471808}
+TRAFFIC = {"tc_gemm_sha1": "1fca5db76d4c8575304b020d1997996562109ab8", "bytes_per_launch": 1141020928}
 
 
 def load_peaks():
@@ -71,8 +71,12 @@ def fractions(tflops, peaks, regime):
 
 
 def kernel_sha1():
-    with open(os.path.join(ROOT, "paper_2401_11504_b200", "csrc", "tc_gemm.cu"), "rb") as f:
-        return hashlib.sha1(f.read()).hexdigest()
+    """Fingerprint of the dominant kernel's source: tc_gemm.cu and the instruction wrappers it is written with."""
+    h = hashlib.sha1()
+    for name in ("tc_gemm.cu", "tc_device.cuh"):
+        with open(os.path.join(ROOT, "paper_2401_11504_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 def main_kernel_flops(projections, T, r):

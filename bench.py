@@ -390,6 +390,8 @@ def run_ours(args):
         torch.cuda.empty_cache()
         extra["config4"] = config_70b(b, torch, inputs, runtime, dev, peaks, hp)
         torch.cuda.empty_cache()
+        extra["mlp"] = mlp_update(b, torch, inputs, runtime, dev, peaks, hp)
+        torch.cuda.empty_cache()
 
     cpu = None
     if ranks.world == 1 and not args.no_cpu_baseline:
@@ -431,6 +433,8 @@ def run_only(args):
     hp = {k: float(v) for k, v in inputs.ADAMW.items()}
     if args.only == "block_ops":
         out = block_ops_bandwidth(b, torch, inputs, dev, peaks, reps=1 if args.steps is None else args.steps)
+    elif args.only == "mlp":
+        out = mlp_update(b, torch, inputs, runtime, dev, peaks, hp)
     elif args.only == "decode":
         out = decode_bandwidth(b, torch, inputs, dev, peaks, n_blocks=args.decode_blocks)
     elif args.only == "config2":
@@ -601,6 +605,71 @@ def _parallel_deployment(b, torch, runtime, blk, hp, update_sms, decode_sms, n_u
         dep.close()
 
 
+def mlp_update(b, torch, inputs, runtime, dev, peaks, hp, T=1024, r=64, steps=40, warmup=5, n_rot=3):
+    """templora_update_mlp on the 7B block's MLP (gate, up 4096 -> 11008, down 11008 -> 4096; T = 1024): gate and up as
+    one GEMM whose epilogue writes gate, up and h = SiLU(gate) * up, dgate and dup written by the epilogue of the down
+    projection's input gradient.  Beside it: what the stand-alone gating kernels take at the same shape (the two
+    [T, d_ff] round trips the fused call does not make) and how many of them the timed calls launched (none)."""
+    d, d_ff, s = 4096, 11008, 2.0
+    projs = [("gate", d, d_ff), ("up", d, d_ff), ("down", d_ff, d)]
+    sets = []
+    for i in range(n_rot):
+        blk = runtime.Block(b, 0, f"mlp{i}", projs, T, r, s, "bf16", dev, with_dX=False)
+        bufs = dict(x=blk.x[0], dY=blk.dY[2], y=blk.y[2],
+                    gate=torch.empty((T, d_ff), dtype=torch.bfloat16, device=dev),
+                    up=torch.empty((T, d_ff), dtype=torch.bfloat16, device=dev),
+                    h=torch.empty((T, d_ff), dtype=torch.bfloat16, device=dev),
+                    dX=torch.empty((T, d), dtype=torch.bfloat16, device=dev))
+        sets.append((blk, bufs))
+    ws = b.alloc_workspace(b.templora_update_mlp_workspace_bytes(sets[0][0].lins, T), dev)
+    step = [0] * n_rot
+
+    def one(i):
+        blk, q = sets[i % n_rot]
+        step[i % n_rot] = b.templora_update_mlp(blk.lins, blk.A_desc, blk.B_desc, q["x"], q["dY"], q["gate"], q["up"], q["h"],
+                                                q["y"], q["dX"], 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                                hp["weight_decay"], step[i % n_rot], ws)
+    for i in range(warmup):
+        one(i)
+    torch.cuda.synchronize()
+    b.templora_timing_enable(False)
+    for k in range(b.N_KINDS):
+        b.templora_timing_read(k, reset=True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with runtime.ClockSampler(torch.cuda.current_device()) as clk:
+        e0.record()
+        for i in range(steps):
+            one(i)
+        e1.record()
+        torch.cuda.synchronize()
+    clocks = clk.summary()
+    assert b.templora_read_device_status(ws)[0] == 0
+    launches = {k: b.templora_timing_read(k)[2] for k in range(b.N_KINDS)}
+    sec = e0.elapsed_time(e1) / 1e3 / steps
+    flops = block_flops(projs, T, r)
+    # the stand-alone gating kernels at this shape, for scale
+    g = sets[0][1]
+    scratch = [torch.empty((T, d_ff), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    def timed(fn, reps=20):
+        fn(); torch.cuda.synchronize()
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        c.record(); torch.cuda.synchronize()
+        return a.elapsed_time(c) / reps * 1e3
+    fwd_us = timed(lambda: b.templora_swiglu_fwd(g["gate"], g["up"], scratch[0]))
+    bwd_us = timed(lambda: b.templora_swiglu_bwd(g["gate"], g["up"], g["h"], scratch[0], scratch[1]))
+    regime = pick_regime(sec * steps, clocks)
+    return {"workload": f"MLP of a llama2_7b block (gate, up {d}->{d_ff}, down {d_ff}->{d}), T={T}, r={r}, one "
+                        "templora_update_mlp call per step (forward, backward, AdamW on the six LoRA matrices)",
+            "steps": steps, "ms_per_step": sec * 1e3, "tokens_per_s": T / sec, "tflops": flops / sec / 1e12,
+            **fractions(flops / sec / 1e12, peaks, regime), "regime": regime,
+            "gating_kernel_launches_in_timed_calls": int(launches[b.KIND_BLOCK_OPS]),
+            "standalone_gating_us_at_this_shape": {"swiglu_fwd": fwd_us, "swiglu_bwd": bwd_us},
+            "launches_per_step": sum(launches.values()) / steps, "clocks": clocks}
+
+
 def block_ops_bandwidth(b, torch, inputs, dev, peaks, T=4096, reps=20):
     """HBM throughput of the SiLU-gating and RMSNorm kernels at 7B widths (bf16; T rows of 11008 for the
     gating, 4 T rows of 4096 for the norm so that a launch outlasts the host's call overhead; four buffer
@@ -757,7 +826,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parallel", action="store_true", help="skip the parallelized-deployment measurement")
     ap.add_argument("--no-configs", action="store_true", help="skip the 32-block stack and the 70B block")
-    ap.add_argument("--only", default=None, choices=["block_ops", "decode", "config2", "config4"],
+    ap.add_argument("--only", default=None, choices=["block_ops", "decode", "config2", "config4", "mlp"],
                     help="run one side measurement alone and print its JSON object (profiling aid; not the bench line)")
     args = ap.parse_args()
     reference = args.impl == "reference"

@@ -133,3 +133,13 @@ def test_lr_at_step_host_function(b):
     for step, w in ((1, 8), (4, 8), (8, 8), (9, 8), (5, 0), (0, 4)):
         got = b.templora_lr_at_step(lr, step, w)
         assert got == float(np.float32(orc.lr_at_step(lr, step, w)))
+
+
+def test_sm_partition_argument_errors_need_no_device(b):
+    # refused before any driver call: nothing to split into, nowhere to put the result, nothing to destroy
+    part = b.SmPartition()
+    assert b.lib.templora_sm_partition_create(0, C.byref(part)) == b.ERR_INVALID_ARG
+    assert b.lib.templora_sm_partition_create(32, None) == b.ERR_INVALID_ARG
+    assert part.handle is None and part.stream_first is None and part.sms_first == 0
+    assert b.lib.templora_sm_partition_destroy(C.byref(part)) == b.ERR_INVALID_ARG
+    assert b.lib.templora_sm_partition_destroy(None) == b.ERR_INVALID_ARG

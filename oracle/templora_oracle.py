@@ -40,9 +40,11 @@ against a hand case built from the first of those vectors and against a scalar
 restatement of the rule with 64-bit seeds and offsets and rows that start inside
 a block.
 
-Parity with numbers printed by the paper: parity unpinned.  The paper prints no
-worked numeric example and no per-layer value for this path; the pins above are
-mathematical.
+Every function of this file has at least one such pin; none is left unpinned.
+The paper itself prints no worked numeric example and no per-layer value for
+this path, so no pin compares with a number printed there: the pins are what the
+mathematics fixes (closed forms, brute force, exact finite differences, textbook
+special cases, a published generator's known answers).
 """
 import numpy as np
 

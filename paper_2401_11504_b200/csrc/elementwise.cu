@@ -24,12 +24,26 @@ __global__ void __launch_bounds__(kRedThreads) reduce_partials_kernel(const __gr
   if (i0 >= jb.n) return;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   const bool vec = (i0 + 4 <= jb.n) && ((jb.stride & 3) == 0) && ((reinterpret_cast<uintptr_t>(jb.part) & 15) == 0);
-  for (int k = 0; k < jb.n_parts; ++k) {
-    const float *p = jb.part + (long long)k * jb.stride + i0;
-    if (vec) {
-      float4 t = *reinterpret_cast<const float4 *>(p);
+  if (vec) {
+    // four slabs' loads are issued before any is added (the sum still runs in slab order): one memory round trip
+    // per four slabs instead of one per slab
+    int k = 0;
+    for (; k + 4 <= jb.n_parts; k += 4) {
+      const float *p = jb.part + (long long)k * jb.stride + i0;
+      const float4 t0 = *reinterpret_cast<const float4 *>(p), t1 = *reinterpret_cast<const float4 *>(p + jb.stride),
+                   t2 = *reinterpret_cast<const float4 *>(p + 2 * jb.stride), t3 = *reinterpret_cast<const float4 *>(p + 3 * jb.stride);
+      acc[0] += t0.x; acc[1] += t0.y; acc[2] += t0.z; acc[3] += t0.w;
+      acc[0] += t1.x; acc[1] += t1.y; acc[2] += t1.z; acc[3] += t1.w;
+      acc[0] += t2.x; acc[1] += t2.y; acc[2] += t2.z; acc[3] += t2.w;
+      acc[0] += t3.x; acc[1] += t3.y; acc[2] += t3.z; acc[3] += t3.w;
+    }
+    for (; k < jb.n_parts; ++k) {
+      const float4 t = *reinterpret_cast<const float4 *>(jb.part + (long long)k * jb.stride + i0);
       acc[0] += t.x; acc[1] += t.y; acc[2] += t.z; acc[3] += t.w;
-    } else {
+    }
+  } else {
+    for (int k = 0; k < jb.n_parts; ++k) {
+      const float *p = jb.part + (long long)k * jb.stride + i0;
       for (int e = 0; e < 4; ++e)
         if (i0 + e < jb.n) acc[e] += p[e];
     }

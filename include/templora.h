@@ -142,7 +142,10 @@ templora_status_t templora_adamw_step(const templora_param_t *params, int32_t n_
 /*
  * Decode-time forward with the current (un-merged) module for n_tokens in 1..16 rows
  * (generation step Y[i] = Theta_k(...) of Algorithm 1):  y = x W0^T + s (x A^T) B^T.
- * Streams W0 once per call; bound by HBM bandwidth.
+ * Streams W0 once per call; bound by HBM bandwidth.  On the tensor-core path the call is one kernel launch
+ * whose counters and flags in the workspace head are re-armed on the device, so after one call outside a
+ * capture (one-time set-up per device and kernel) it, and templora_decode_block_fwd, may be recorded into a CUDA
+ * graph and replayed with new contents in the same x buffer.
  */
 templora_status_t templora_decode_fwd(const templora_linear_t *lin, int32_t n_tokens, const void *x, void *y,
                                       void *ws, size_t ws_bytes, void *stream);

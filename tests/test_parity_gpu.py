@@ -449,8 +449,8 @@ def test_decode_two_kernel_form(b, n):
 
 
 def test_decode_repeated_calls_share_a_workspace(b):
-    # s*u of an earlier call stays in the workspace; every call must wait for its own (ready flags carry
-    # a per-launch number) and the item counter must be re-armed between calls, also across the two forms
+    # s*u of an earlier call stays in the workspace; every call must wait for its own (the ready flags are
+    # cleared at the end of each launch) and the item counter must be re-armed between calls, also across the two forms
     d_in, d_out, r = 4096, 1280, 64
     host = inputs.make_linear(22, "dec-rep", 16, d_in, d_out, r, dtype="bf16")
     lin_probe = b.linear_desc(host["W0"].cuda(), host["A"].cuda(), host["B"].cuda(), 2.0)
@@ -462,6 +462,42 @@ def test_decode_repeated_calls_share_a_workspace(b):
             _decode_case(b, 23 + rep, f"dec-rep-{rep}", (1, 16, 4, 7, 2, 16)[rep], d_in, d_out, r, ws=ws)
         finally:
             b.templora_set_kernel_path(0)
+
+
+def test_decode_block_replayed_from_a_cuda_graph(b):
+    # the launch depends on nothing the host hands in per call (ready flags and the item counter are re-armed on the
+    # device), so a decode step recorded once can be replayed: new inputs in the same buffers, same results as a
+    # direct call and as the oracle
+    shapes = [(1024, 768, 64), (1024, 768, 64), (768, 1024, 32)]
+    n = 4
+    hosts = [inputs.make_linear(61, f"graph{i}", n, di, do, r, dtype="bf16") for i, (di, do, r) in enumerate(shapes)]
+    devs = [{k: v.cuda() for k, v in h.items()} for h in hosts]
+    lins = [b.linear_desc(d["W0"], d["A"], d["B"], 2.0) for d in devs]
+    xs = [d["x"].clone() for d in devs]
+    ys = [torch.empty((n, do), dtype=torch.bfloat16, device="cuda") for _, do, _ in shapes]
+    ws = b.alloc_workspace(b.templora_decode_block_workspace_bytes(lins))
+    args = b.DecodeBlockArgs(lins, xs, ys)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        b.templora_decode_block_fwd(args, ws, stream=side)      # first call outside the capture: one-time set-up
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        b.templora_decode_block_fwd(args, ws, stream=torch.cuda.current_stream())
+    for rep in range(3):
+        new_x = [inputs.make_tensor(62 + rep, f"graph{i}", "x", (n, di), "normal", 1.0, "bf16", "cpu") for i, (di, _, _) in enumerate(shapes)]
+        for x, nx in zip(xs, new_x):
+            x.copy_(nx.cuda())
+        for y in ys:
+            y.fill_(float("nan"))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert b.templora_read_device_status(ws)[0] == 0
+        for i, h in enumerate(hosts):
+            ref = orc.decode_fwd(f64(new_x[i]), f64(h["W0"]), f64(h["A"]), f64(h["B"]), 2.0)
+            assert_close(f"graph replay {rep} y{i}", f64(ys[i]), ref, TOL["bf16"])
 
 
 # ------------------------------------------------------------------ projections that share their input

@@ -278,6 +278,30 @@ templora_status_t templora_update_mlp(const templora_linear_t *proj, const templ
                                       void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * The chunk update of the projections that read a decoder block's normalised input, in one call (the training
+ * step of Theta_k, Algorithm 1, run over RMSNorm -> q, k, v of a Llama-style block; the norm is the model's, its
+ * weight frozen):
+ *     xn  = RMSNorm(x; norm_weight, norm_eps)                          (as templora_rmsnorm_fwd)
+ *     y_i = xn W_i^T + s_i (xn A_i^T) B_i^T                            i = 0 .. n_proj-1, n_proj <= 3
+ * and, from the dY_i:
+ *     dXn = sum_i (dY_i W_i + s_i (dY_i B_i) A_i)      ONE summed gradient with respect to xn, formed in the
+ *                                                      accumulator of one GEMM (as templora_linear_t.input_group)
+ *     dX  = RMSNorm backward of dXn                                    (as templora_rmsnorm_bwd)
+ * with the LoRA gradients as in templora_linear_bwd and one AdamW step on all A_i, B_i; `epochs` times (x does not
+ * change between epochs, so xn is formed once; dXn and dX are the last epoch's).
+ *   proj, A_state, B_state: HOST arrays of n_proj entries, aliased as in templora_update_block; equal d_in and dtype
+ *   (input_group is ignored: the projections share their input by construction).  dY, y: HOST arrays of n_proj
+ *   device pointers.  x [T, d_in], norm_weight [d_in] inputs; xn, dXn [T, d_in] outputs; dX [T, d_in] output or NULL.
+ *   Workspace: templora_update_block_workspace_bytes(proj, n_proj, T).
+ */
+templora_status_t templora_update_attn_in(const templora_linear_t *proj, const templora_param_t *A_state,
+                                          const templora_param_t *B_state, int32_t n_proj, int32_t T, const void *x,
+                                          const void *norm_weight, float norm_eps, const void *const *dY, void *xn,
+                                          void *const *y, void *dXn, void *dX, int32_t epochs, float lr, float beta1,
+                                          float beta2, float eps, float weight_decay, int64_t *step_inout, void *ws,
+                                          size_t ws_bytes, void *stream);
+
+/*
  * Failure-detection self-test (the paper has no counterpart).  Enqueues one tiny kernel that
  * waits, the way the GEMM kernels wait for their copies, on a barrier that nothing signals.
  * After limit_ms (1..1000) it records TEMPLORA_ERR_TIMEOUT in the status record at the head of

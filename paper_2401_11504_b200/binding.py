@@ -26,6 +26,7 @@ EXPORTS = [
     "templora_update_block_warmup", "templora_swiglu_fwd", "templora_swiglu_bwd", "templora_rmsnorm_fwd",
     "templora_rmsnorm_bwd", "templora_decode_fwd_noalloc_status", "templora_update_mlp",
     "templora_update_mlp_workspace_bytes", "templora_sm_partition_create", "templora_sm_partition_destroy",
+    "templora_update_attn_in",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 (KIND_TC_MAIN, KIND_TC_SKINNY, KIND_TC_DECODE, KIND_REDUCE, KIND_ADAMW, KIND_SIMT, KIND_DECODE_FINISH, KIND_DROPOUT,
@@ -90,6 +91,9 @@ def _load():
     lib.templora_update_mlp.restype = i32
     lib.templora_update_mlp.argtypes = [LP, PP, PP, i32, vp, vp, vp, vp, vp, vp, vp, i32, f32, f32, f32, f32, f32,
                                         C.POINTER(i64), vp, sz, vp]
+    lib.templora_update_attn_in.restype = i32
+    lib.templora_update_attn_in.argtypes = [LP, PP, PP, i32, i32, vp, vp, f32, C.POINTER(vp), vp, C.POINTER(vp), vp, vp,
+                                            i32, f32, f32, f32, f32, f32, C.POINTER(i64), vp, sz, vp]
     lib.templora_swiglu_fwd.restype = i32
     lib.templora_swiglu_fwd.argtypes = [i64, i32, vp, vp, vp, vp]
     lib.templora_swiglu_bwd.restype = i32
@@ -281,6 +285,22 @@ def templora_update_mlp(lins, A_states, B_states, x, dY, gate, up, h, y, dX, epo
                                    x.shape[0], _ptr(x), _ptr(dY), _ptr(gate), _ptr(up), _ptr(h), _ptr(y), _ptr(dX),
                                    int(epochs), lr, beta1, beta2, eps, weight_decay, C.byref(st), _ptr(ws), ws.numel(),
                                    _stream(stream)), "templora_update_mlp")
+    return st.value
+
+
+def templora_update_attn_in(lins, A_states, B_states, x, norm_weight, norm_eps, dYs, xn, ys, dXn, dX, epochs, lr, beta1,
+                            beta2, eps, weight_decay, step, ws, stream=None):
+    """Chunk update of the projections behind a block's input norm (q, k, v): RMSNorm, the projections on the shared
+    normalised input with one summed input gradient, the norm's backward; returns the new step count."""
+    n = len(lins)
+    st = C.c_int64(int(step))
+    vp = C.c_void_p
+    dy_arr = (vp * n)(*[t.data_ptr() for t in dYs])
+    y_arr = (vp * n)(*[t.data_ptr() for t in ys])
+    _check(lib.templora_update_attn_in((LinearDesc * n)(*lins), (ParamDesc * n)(*A_states), (ParamDesc * n)(*B_states), n,
+                                       x.shape[0], _ptr(x), _ptr(norm_weight), norm_eps, dy_arr, _ptr(xn), y_arr, _ptr(dXn),
+                                       _ptr(dX), int(epochs), lr, beta1, beta2, eps, weight_decay, C.byref(st), _ptr(ws),
+                                       ws.numel(), _stream(stream)), "templora_update_attn_in")
     return st.value
 
 

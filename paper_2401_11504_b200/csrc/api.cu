@@ -1316,6 +1316,43 @@ templora_status_t templora_update_mlp(const templora_linear_t *proj, const templ
                   step_inout, ws, ws_bytes, false, nullptr, reinterpret_cast<cudaStream_t>(stream));
 }
 
+templora_status_t templora_update_attn_in(const templora_linear_t *proj, const templora_param_t *A_state,
+                                          const templora_param_t *B_state, int32_t n_proj, int32_t T, const void *x,
+                                          const void *norm_weight, float norm_eps, const void *const *dY, void *xn,
+                                          void *const *y, void *dXn, void *dX, int32_t epochs, float lr, float beta1,
+                                          float beta2, float eps, float weight_decay, int64_t *step_inout, void *ws,
+                                          size_t ws_bytes, void *stream) {
+  if (!proj || n_proj < 1 || n_proj > 3 || T <= 0 || !x || !norm_weight || !dY || !xn || !y || !dXn) return TEMPLORA_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(norm_weight) || !aligned16(xn) || !aligned16(dXn) || (dX && !aligned16(dX)))
+    return TEMPLORA_ERR_INVALID_ARG;
+  if (!(norm_eps >= 0.f)) return TEMPLORA_ERR_INVALID_ARG;
+  // the projections read ONE tensor (the normalised input) and their input gradients are summed into ONE buffer
+  templora_linear_t shared[3];
+  const void *xs[3];
+  void *dXs[3];
+  for (int i = 0; i < n_proj; ++i) {
+    TL_TRY(check_linear(proj + i));
+    if (proj[i].d_in != proj[0].d_in || proj[i].dtype != proj[0].dtype) return TEMPLORA_ERR_INVALID_ARG;
+    shared[i] = proj[i];
+    shared[i].input_group = 1;
+    xs[i] = xn;
+    dXs[i] = dXn;
+  }
+  const int d = proj[0].d_in, dt = proj[0].dtype;
+  // every argument check of the update runs before anything is enqueued (zero epochs: checks only)
+  {
+    int64_t probe = step_inout ? *step_inout : 0;
+    TL_TRY(templora_update_block(shared, A_state, B_state, n_proj, T, xs, dY, y, dXs, 0, lr, beta1, beta2, eps,
+                                 weight_decay, step_inout ? &probe : nullptr, ws, ws_bytes, stream));
+    if (epochs < 0) return TEMPLORA_ERR_INVALID_ARG;
+  }
+  TL_TRY(templora_rmsnorm_fwd(T, d, dt, x, norm_weight, norm_eps, xn, stream));
+  TL_TRY(templora_update_block(shared, A_state, B_state, n_proj, T, xs, dY, y, dXs, epochs, lr, beta1, beta2, eps,
+                               weight_decay, step_inout, ws, ws_bytes, stream));
+  if (dX && epochs > 0) TL_TRY(templora_rmsnorm_bwd(T, d, dt, x, norm_weight, dXn, norm_eps, dX, stream));
+  return TEMPLORA_OK;
+}
+
 const char *templora_status_string(templora_status_t st) {
   switch (st) {
     case TEMPLORA_OK: return "ok";
